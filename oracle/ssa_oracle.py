@@ -1,0 +1,298 @@
+"""Plain fp64 CPU statement of span-restricted decode attention.
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg; never by the product path.  It shares no code
+with the CUDA library (own storage decoders, own status constants).
+
+What is stated here, and where the paper defines it:
+
+* ``spans_to_index``      the set of context positions a request may attend
+                          to, as the sorted list of positions covered by its
+                          token spans (Sec. "Self-selected attention span":
+                          groups of contiguous tokens; Sec. "CUDA Kernel
+                          Design": the span may be non-contiguous, and a
+                          per-token binary mask records what is attended).
+* ``attn_set_form``       masked attention for the single query row of a
+                          decode step (Background, equations for S, A and O;
+                          "Token generation": one row of S and A per step),
+                          with the mask 0 on the selected set and -inf
+                          elsewhere.
+* ``attn_dense``          the same with every position kept.
+* ``attn_additive_mask``  the background equations taken literally: all
+                          scores, plus a 0/-inf mask, softmax, times V.
+* ``attn_alg1_blocked``   Algorithm 1 (blocked span encoding: block index +
+                          block bitmask, empty blocks omitted) with the
+                          readings listed below.
+* ``merge_partials``      recombination of (max, sum, accumulator) partial
+                          results of disjoint subsets; not in the paper (its
+                          kernel runs one thread block per head and request),
+                          it is the algebra of the softmax itself.
+
+Readings of Algorithm 1 where its printed form cannot be taken literally:
+  - the mask conversion on the block bitmask is read from the prose next to
+    it: bit 1 adds 0 to the score, bit 0 adds -inf;
+  - scores of blocks absent from the metadata are -inf (the text says
+    attention is computed only over the selected span), not the initial 0;
+  - the output is a d-vector accumulated over all selected tokens
+    (O = A V), not an n-vector assigned per token;
+  - whether the metadata holds a bitmask or start/end offsets inside the
+    block is immaterial to the result; the bitmask form is used.
+The softmax scale is exposed as an argument; callers pass 1/sqrt(head_dim).
+An empty selection (never produced by the method, which always keeps the
+instruction and the previous line) yields a zero row and lse = -inf.
+
+Pins (tests marked "not gpu"): hand-enumerated index lists and a set
+brute force; the worked anchor/reference examples of the paper as span
+structure; closed forms of the softmax (one token, two tokens, uniform
+weights, weights 1/6 2/6 3/6); agreement of the three formulations above;
+a library scaled-dot-product attention in fp64; convexity, shift, permutation
+and split/merge invariants; independence from unselected rows.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+# Status bits a span list can raise (diagnostics; the index list itself always
+# follows the set definition).
+ST_BAD_SPAN = 1    # start < 0 or start > end
+ST_CLIPPED = 2     # end > context length
+ST_OVERFLOW = 4    # more selected positions than the index row can hold
+
+
+# --------------------------------------------------------------------------
+# storage decoders (16-bit patterns -> float64, exact)
+# --------------------------------------------------------------------------
+def decode_bits(u16, dtype: str) -> np.ndarray:
+    """Exact value of 16-bit storage patterns as float64.
+
+    ``bf16``: the pattern is the upper half of an IEEE binary32.
+    ``f16`` : IEEE binary16.
+    """
+    a = np.ascontiguousarray(u16)
+    if a.dtype != np.uint16:
+        raise TypeError("expected uint16 bit patterns")
+    if dtype == "bf16":
+        with np.errstate(invalid="ignore"):      # signalling NaN patterns
+            return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    if dtype == "f16":
+        return a.view(np.float16).astype(np.float64)
+    raise ValueError(f"unknown storage dtype {dtype!r}")
+
+
+# --------------------------------------------------------------------------
+# spans -> index list
+# --------------------------------------------------------------------------
+def spans_to_index(spans, n: int) -> np.ndarray:
+    """Sorted positions j in [0, n) covered by at least one span [s, e).
+
+    Definition by marking: a per-position boolean "may attend" array is
+    filled span by span and the marked positions are emitted in increasing
+    order.  Order, overlap and repetition of spans therefore cannot matter.
+    """
+    n = int(n)
+    mark = np.zeros(max(n, 0), dtype=bool)
+    for s, e in np.asarray(spans, dtype=np.int64).reshape(-1, 2):
+        lo = max(int(s), 0)
+        hi = min(int(e), n)
+        if hi > lo:
+            mark[lo:hi] = True
+    return np.flatnonzero(mark).astype(np.int32)
+
+
+def spans_status(spans, n: int, index_stride: int | None = None) -> int:
+    """Diagnostic bits for one request's span list (see ST_* above)."""
+    st = 0
+    for s, e in np.asarray(spans, dtype=np.int64).reshape(-1, 2):
+        if s < 0 or s > e:
+            st |= ST_BAD_SPAN
+        if e > n:
+            st |= ST_CLIPPED
+    if index_stride is not None and len(spans_to_index(spans, n)) > index_stride:
+        st |= ST_OVERFLOW
+    return st
+
+
+def spans_to_index_batch(span_offsets, spans, ctx_lens, index_stride: int):
+    """Batch form with the padded row layout of the library interface.
+
+    Returns (index[B, index_stride] int32 filled with -1 past the count,
+    counts[B] int32, status bits OR-ed over the batch).  A request whose list
+    is longer than ``index_stride`` keeps its first ``index_stride`` positions.
+    """
+    span_offsets = np.asarray(span_offsets, dtype=np.int64)
+    spans = np.asarray(spans, dtype=np.int64).reshape(-1, 2)
+    B = len(ctx_lens)
+    index = np.full((B, index_stride), -1, dtype=np.int32)
+    counts = np.zeros(B, dtype=np.int32)
+    status = 0
+    for b in range(B):
+        sp = spans[span_offsets[b]:span_offsets[b + 1]]
+        idx = spans_to_index(sp, int(ctx_lens[b]))
+        status |= spans_status(sp, int(ctx_lens[b]), index_stride)
+        c = min(len(idx), index_stride)
+        index[b, :c] = idx[:c]
+        counts[b] = c
+    return index, counts, status
+
+
+# --------------------------------------------------------------------------
+# attention for one (request, head): q[D], K[n, D], V[n, D] in float64
+# --------------------------------------------------------------------------
+def attn_partial(q, K, V, idx, scale: float):
+    """(m, l, acc) over the positions ``idx``: m = max score,
+    l = sum exp(score - m), acc[d] = sum exp(score - m) V[j, d]."""
+    idx = np.asarray(idx, dtype=np.int64)
+    D = V.shape[-1]
+    if idx.size == 0:
+        return -np.inf, 0.0, np.zeros(D)
+    s = scale * (K[idx] @ q)
+    m = float(np.max(s))
+    w = np.exp(s - m)
+    return m, float(np.sum(w)), w @ V[idx]
+
+
+def attn_set_form(q, K, V, idx, scale: float):
+    """out[d] = sum_j softmax_j(scale q.K_j) V[j, d] over j in ``idx``;
+    lse = log sum_j exp(scale q.K_j).  Rows outside ``idx`` are never read."""
+    m, l, acc = attn_partial(q, K, V, idx, scale)
+    if l == 0.0:
+        return np.zeros(V.shape[-1]), -np.inf
+    return acc / l, m + np.log(l)
+
+
+def attn_dense(q, K, V, n: int, scale: float):
+    """Every position 0..n-1 kept (the full-context step)."""
+    D = V.shape[-1]
+    if n <= 0:
+        return np.zeros(D), -np.inf
+    s = (K[:n] @ q) * scale
+    m = np.max(s)
+    a = np.exp(s - m)
+    z = np.sum(a)
+    return (a / z) @ V[:n], float(m + np.log(z))
+
+
+def attn_additive_mask(q, K, V, n: int, keep, scale: float):
+    """The background equations as printed: S = qK^T scaled, M is 0 where
+    attention is permitted and -inf where it is prohibited, A = softmax(M+S),
+    O = A V.  ``keep`` is a boolean array over the n positions."""
+    keep = np.asarray(keep, dtype=bool)[:n]
+    S = (K[:n] @ q) * scale
+    M = np.where(keep, 0.0, -np.inf)
+    Z = M + S
+    zmax = np.max(Z) if n > 0 else -np.inf
+    if not np.isfinite(zmax):
+        return np.zeros(V.shape[-1]), -np.inf
+    E = np.exp(Z - zmax)
+    A = E / np.sum(E)
+    return A @ V[:n], float(zmax + np.log(np.sum(E)))
+
+
+def encode_blocked(idx, bs: int):
+    """Blocked span encoding: for every block of ``bs`` consecutive positions
+    holding at least one selected position, (block index, bs-bit mask of the
+    selected positions inside it); empty blocks are omitted."""
+    meta = {}
+    for j in np.asarray(idx, dtype=np.int64):
+        blk, off = divmod(int(j), bs)
+        meta.setdefault(blk, np.zeros(bs, dtype=bool))[off] = True
+    return [(blk, meta[blk]) for blk in sorted(meta)]
+
+
+def attn_alg1_blocked(q, K, V, n: int, metadata, bs: int, scale: float):
+    """Algorithm 1 with the readings stated in the module header."""
+    D = V.shape[-1]
+    nb = (max(n, 0) + bs - 1) // bs
+    qK = np.full(nb * bs, -np.inf)            # unlisted blocks: excluded
+    for blk, bm in metadata:
+        soft = np.where(bm, 0.0, -np.inf)     # bit 1 -> +0, bit 0 -> -inf
+        delta = blk * bs
+        bqK = np.zeros(bs)
+        for i in range(bs):
+            if delta + i < n:
+                bqK[i] = float(np.dot(q, K[delta + i]))
+        qK[delta:delta + bs] = bqK + soft
+    Z = qK * scale
+    zmax = np.max(Z) if Z.size else -np.inf
+    if not np.isfinite(zmax):
+        return np.zeros(D), -np.inf
+    E = np.exp(Z - zmax)
+    A = E / np.sum(E)
+    o = np.zeros(D)
+    for blk, bm in metadata:
+        delta = blk * bs
+        for i in range(bs):
+            if delta + i < n and A[delta + i] != 0.0:
+                o += A[delta + i] * V[delta + i]
+    return o, float(zmax + np.log(np.sum(E)))
+
+
+def merge_partials(ms, ls, accs):
+    """Combine partial results of disjoint position subsets:
+    m = max m_k, l = sum l_k e^(m_k - m), out = sum acc_k e^(m_k - m) / l."""
+    ms = np.asarray(ms, dtype=np.float64)
+    ls = np.asarray(ls, dtype=np.float64)
+    accs = np.asarray(accs, dtype=np.float64)
+    m = np.max(ms) if ms.size else -np.inf
+    if not np.isfinite(m):
+        return np.zeros(accs.shape[-1]), -np.inf
+    f = np.where(np.isfinite(ms), np.exp(ms - m), 0.0)
+    l = float(np.sum(ls * f))
+    return (f[:, None] * accs).sum(axis=0) / l, float(m + np.log(l))
+
+
+# --------------------------------------------------------------------------
+# batch forms over a KV cache (logical layout [B, H, T, D])
+# --------------------------------------------------------------------------
+def _as_f64(a, dtype):
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return decode_bits(a, dtype)
+    return a.astype(np.float64)
+
+
+def decode_attn_sparse(q, k_cache, v_cache, ctx_lens, index, counts, scale,
+                       dtype: str = "bf16", heads=None, seqs=None):
+    """Span-restricted decode attention for a batch.
+
+    q[B, H, D]; k_cache, v_cache[B, H, T, D] (uint16 storage patterns of
+    ``dtype`` or floats; any numpy strides); index[B, stride] with counts[B]
+    valid entries per request, shared by all heads of the request.  Entries
+    outside [0, ctx_lens[b]) are skipped.  ``seqs`` / ``heads`` restrict the
+    work to a sample; untouched rows of the result are NaN.
+    Returns out[B, H, D] float64 and lse[B, H] float64.
+    """
+    B, H, D = q.shape
+    out = np.full((B, H, D), np.nan)
+    lse = np.full((B, H), np.nan)
+    for b in (range(B) if seqs is None else seqs):
+        n = int(ctx_lens[b])
+        idx = np.asarray(index[b][: int(counts[b])], dtype=np.int64)
+        idx = idx[(idx >= 0) & (idx < n)]
+        for h in (range(H) if heads is None else heads):
+            qv = _as_f64(q[b, h], dtype)
+            # decode only the gathered rows; the others are never touched
+            Ks = _as_f64(np.asarray(k_cache[b, h])[idx], dtype)
+            Vs = _as_f64(np.asarray(v_cache[b, h])[idx], dtype)
+            o, e = attn_set_form(qv, Ks, Vs, np.arange(len(idx)), scale)
+            out[b, h] = o
+            lse[b, h] = e
+    return out, lse
+
+
+def decode_attn_dense(q, k_cache, v_cache, ctx_lens, scale,
+                      dtype: str = "bf16", heads=None, seqs=None):
+    """Full-context decode attention for a batch (same conventions)."""
+    B, H, D = q.shape
+    out = np.full((B, H, D), np.nan)
+    lse = np.full((B, H), np.nan)
+    for b in (range(B) if seqs is None else seqs):
+        n = int(ctx_lens[b])
+        for h in (range(H) if heads is None else heads):
+            qv = _as_f64(q[b, h], dtype)
+            Kf = _as_f64(np.asarray(k_cache[b, h])[:n], dtype)
+            Vf = _as_f64(np.asarray(v_cache[b, h])[:n], dtype)
+            o, e = attn_dense(qv, Kf, Vf, n, scale)
+            out[b, h] = o
+            lse[b, h] = e
+    return out, lse
