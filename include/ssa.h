@@ -1,0 +1,199 @@
+/*
+ * ssa.h - span-restricted ("self-selected attention span") decode attention
+ *         for NVIDIA B200 (sm_100a).  C ABI of libssa.
+ *
+ * One decode step of the method: every request of a batch attends, with its
+ * single query row per head, only to the KV-cache rows of the token spans
+ * currently selected for it (Sec. "Self-selected attention span", "Token
+ * generation"; Sec. "CUDA Kernel Design").  The result is exactly masked
+ * attention (Background: S = q K^T / sqrt(d), A = softmax(M + S), O = A V)
+ * with M = 0 on the selected positions and -inf elsewhere.
+ *
+ * General conventions
+ *  - Every pointer marked "dev" is a DEVICE pointer owned by the caller; the
+ *    library never allocates, frees or keeps device memory between calls.
+ *    Pointers marked "host" are ordinary host pointers read during the call.
+ *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *    the default stream).  No call synchronises or reads device memory back,
+ *    so everything data-dependent (selected counts, context lengths) stays on
+ *    the device and host-side sizes are upper bounds.
+ *  - Return value: an ssa_status.  Non-zero means nothing was launched.
+ *  - Data-dependent problems never fault: they set bits in the caller's
+ *    device status word (`dev_status`, may be NULL) and take the defined
+ *    fallback (clip / skip / truncate).
+ *  - Selection is per request and shared by all heads of the request (the
+ *    paper keeps separate metadata per request of a batch).
+ */
+#ifndef SSA_H_
+#define SSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SSA_OK = 0,
+  SSA_ERR_NULL = 1,        /* a required pointer is NULL                          */
+  SSA_ERR_SHAPE = 2,       /* a size is non-positive or out of the supported range */
+  SSA_ERR_DTYPE = 3,       /* unsupported kv_dtype / out_dtype                     */
+  SSA_ERR_ALIGN = 4,       /* pointer or stride not 16-byte aligned                */
+  SSA_ERR_CAPACITY = 5,    /* index_stride / max_selected inconsistent             */
+  SSA_ERR_WORKSPACE = 6,   /* workspace missing or too small                       */
+  SSA_ERR_CUDA = 7,        /* a CUDA runtime call or launch failed                 */
+  SSA_ERR_UNSUPPORTED = 8  /* valid request outside the implemented set            */
+} ssa_status;
+
+/* Bits OR-ed into *dev_status by kernels. */
+enum {
+  SSA_DEV_BAD_SPAN = 1,    /* a span had start < 0 or start > end                  */
+  SSA_DEV_CLIPPED = 2,     /* a span had end > ctx_len and was clipped             */
+  SSA_DEV_OVERFLOW = 4,    /* a request selected more than index_stride positions;
+                              its list was truncated to the first index_stride     */
+  SSA_DEV_BAD_INDEX = 8,   /* an index entry was outside [0, ctx_len): skipped     */
+  SSA_DEV_BAD_COUNT = 16,  /* counts[b] > max_selected or ctx_lens[b] > max_ctx:
+                              clamped                                              */
+  SSA_DEV_TOO_MANY_SPANS = 32 /* a request had more than SSA_MAX_SPANS_PER_SEQ
+                              spans; the surplus was ignored                       */
+};
+
+#define SSA_MAX_SPANS_PER_SEQ 2048
+
+typedef enum { SSA_F16 = 0, SSA_BF16 = 1, SSA_F32 = 2 } ssa_dtype;
+
+/*
+ * Geometry of q, the KV cache and the output.  Strides are in ELEMENTS; the
+ * head dimension is contiguous in every tensor.  Both the per-head layout
+ * [B, H, T, D] and the token-major layout [B, T, H, D] are expressible.
+ *   q   [b, h, :]    at q   + b*q_stride_b + h*q_stride_h
+ *   K   [b, t, h, :] at k   + b*k_stride_b + t*k_stride_t + h*k_stride_h
+ *   V   likewise with the v_* strides
+ *   out [b, h, :]    at out + b*o_stride_b + h*o_stride_h
+ * Row t = ctx_lens[b]-1 is the current token's own K/V, appended by the
+ * caller before the call; it is attended only if selected.
+ * Supported: D in {64, 128}; kv_dtype F16 or BF16 (q has the same type);
+ * out_dtype equal to kv_dtype or F32; H_kv == H (multi-head attention, as in
+ * the paper's LLaMA-7B).  Every base pointer and every stride * element size
+ * must be a multiple of 16 bytes.
+ */
+typedef struct {
+  int32_t B, H, H_kv, D;
+  int32_t max_ctx;          /* rows allocated per request in the cache            */
+  int32_t kv_dtype;         /* ssa_dtype                                          */
+  int32_t out_dtype;        /* ssa_dtype                                          */
+  float   scale;            /* softmax scale; <= 0 selects 1/sqrt(D)              */
+  int64_t q_stride_b, q_stride_h;
+  int64_t k_stride_b, k_stride_t, k_stride_h;
+  int64_t v_stride_b, v_stride_t, v_stride_h;
+  int64_t o_stride_b, o_stride_h;
+} ssa_attn_desc;
+
+/*
+ * Span list -> compact KV index list (the "on the fly" conversion of the
+ * selected references into an attention mask, Abstract and Sec. "CUDA Kernel
+ * Design", Attention span encoding; here the mask is kept as the sorted list
+ * of attended positions instead of block bitmasks).
+ *
+ * For request b with spans (s_i, e_i), i in [span_offsets[b], span_offsets[b+1]):
+ *   index[b*index_stride + 0 .. counts[b]) = ascending { j : 0 <= j < ctx_lens[b]
+ *                                             and s_i <= j < e_i for some i }.
+ * Spans may be unsorted, overlapping, adjacent, repeated or empty: the result
+ * is the sorted duplicate-free union.  Entries past counts[b] are left
+ * untouched.  start < 0 is clamped to 0 and start > end contributes nothing
+ * (both set SSA_DEV_BAD_SPAN); end > ctx_lens[b] is clipped (SSA_DEV_CLIPPED);
+ * more than index_stride positions keep the first index_stride
+ * (SSA_DEV_OVERFLOW).
+ *
+ *   span_offsets dev int32 [B+1], non-decreasing, span_offsets[0] >= 0
+ *   spans        dev int32 [2 * span_offsets[B]]  (start, end) pairs, 8-byte
+ *                aligned, non-NULL even when there are no spans
+ *   ctx_lens     dev int32 [B]
+ *   index        dev int32 [B * index_stride]     (written)
+ *   counts       dev int32 [B]                    (written)
+ *   dev_status   dev uint32 [1] or NULL           (bits OR-ed in)
+ * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE (B <= 0, B > 65535 or
+ * index_stride <= 0), SSA_ERR_ALIGN, SSA_ERR_CUDA.
+ */
+int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t* spans,
+                           const int32_t* ctx_lens, int32_t B,
+                           int32_t* index, int32_t index_stride,
+                           int32_t* counts, uint32_t* dev_status, void* stream);
+
+/*
+ * Bytes of device workspace the two attention calls need for `desc` when no
+ * request selects more than `max_selected` positions (for the dense call pass
+ * desc->max_ctx).  Returns 0 for an invalid descriptor.  The workspace holds
+ * the per-split partial results (running max, running sum, fp32 accumulator)
+ * of the split-KV pass (the paper's kernel runs one thread block per head and
+ * request and has no such step); its contents need no initialisation and are
+ * dead after the call's work has run.
+ */
+size_t ssa_decode_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selected);
+
+/*
+ * Span-restricted decode attention (Algorithm 1; Background equations with a
+ * 0 / -inf mask): for every request b and head h
+ *   s_j = scale * <q[b,h,:], K[b,j,h,:]>          j in the request's index list
+ *   out[b,h,:] = sum_j softmax_j(s) * V[b,j,h,:]
+ *   lse[b,h]   = log sum_j exp(s_j)               (natural log; optional)
+ * computed with fp32 accumulation.  Only the selected rows of K and V are
+ * read.  The list is index[b*index_stride .. + counts[b]); entries need not be
+ * sorted; a duplicated entry is counted twice; an entry outside
+ * [0, ctx_lens[b]) is skipped (SSA_DEV_BAD_INDEX).  counts[b] == 0 gives a
+ * zero output row and lse = -inf.  `max_selected` is a host-side upper bound
+ * on every counts[b] (1 <= max_selected <= index_stride); a larger count is
+ * clamped to it (SSA_DEV_BAD_COUNT).
+ *
+ *   desc       host
+ *   q, k_cache, v_cache  dev, kv_dtype
+ *   ctx_lens   dev int32 [B]
+ *   index      dev int32 [B * index_stride];  counts dev int32 [B]
+ *   out        dev, out_dtype (written);  lse dev float [B*H] or NULL (written)
+ *   workspace  dev, >= ssa_decode_workspace_bytes(desc, max_selected) bytes,
+ *              16-byte aligned
+ * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE, SSA_ERR_DTYPE, SSA_ERR_ALIGN,
+ * SSA_ERR_CAPACITY, SSA_ERR_WORKSPACE, SSA_ERR_UNSUPPORTED, SSA_ERR_CUDA.
+ */
+int32_t ssa_decode_attn_sparse(const ssa_attn_desc* desc, const void* q,
+                               const void* k_cache, const void* v_cache,
+                               const int32_t* ctx_lens, const int32_t* index,
+                               int32_t index_stride, const int32_t* counts,
+                               int32_t max_selected, void* out, float* lse,
+                               void* workspace, size_t workspace_bytes,
+                               uint32_t* dev_status, void* stream);
+
+/*
+ * Full-context decode attention, the baseline the method is compared with
+ * (Background equations with M = 0; the paper's "determine attention span"
+ * steps attend to all preceding context): as above with the implicit list
+ * 0 .. ctx_lens[b]-1 read as one contiguous stream.  ctx_lens[b] > max_ctx is
+ * clamped (SSA_DEV_BAD_COUNT).  Workspace: ssa_decode_workspace_bytes(desc,
+ * desc->max_ctx).
+ */
+int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q,
+                              const void* k_cache, const void* v_cache,
+                              const int32_t* ctx_lens, void* out, float* lse,
+                              void* workspace, size_t workspace_bytes,
+                              uint32_t* dev_status, void* stream);
+
+/*
+ * Optional timing hook for harnesses (no counterpart in the paper): the next
+ * attention call made by the calling thread records `ev_begin` immediately
+ * before and `ev_end` immediately after its main (split-KV) kernel on the
+ * call's stream, then forgets them.  Both are cudaEvent_t passed as void*;
+ * passing NULLs clears the hook.  Has no effect on results.
+ */
+void ssa_set_kernel_events(void* ev_begin, void* ev_end);
+
+/* Number of kernels the calling thread's calls have launched so far. */
+uint64_t ssa_launch_count(void);
+
+const char* ssa_status_string(int32_t status);
+int32_t ssa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSA_H_ */

@@ -1,0 +1,356 @@
+// Split-KV decode attention over a KV index list (ssa_decode_attn_sparse) or
+// over the full context (ssa_decode_attn_dense).
+//
+// Pass 1 (decode_partial_kernel): grid (chunk, head, request).  A block owns
+// `chunk` consecutive entries of the request's index list (dense: `chunk`
+// consecutive positions).  A cache row of D 16-bit values is read by a group
+// of D/8 lanes with one 16-byte load per lane, so a warp covers 32/(D/8) rows
+// per load instruction and every 32-byte sector of a selected row is fetched
+// exactly once.  Each lane keeps kU K-loads and kU V-loads in flight, then
+// reduces the kU dot products across its lane group with shuffles and folds
+// them into a running (max, sum, accumulator) triple - the online form of the
+// softmax.  Lane groups never talk to one another until the block ends, where
+// their triples are combined through shared memory.  With one chunk per
+// request the block normalises and stores the output itself; otherwise it
+// stores the unnormalised triple to the workspace and
+// Pass 2 (decode_merge_kernel) combines the chunks of one (request, head).
+#include "ssa_common.cuh"
+
+namespace ssa {
+
+#ifndef SSA_WARPS
+#define SSA_WARPS 4
+#endif
+#ifndef SSA_U
+#define SSA_U 8
+#endif
+
+constexpr int kWarps = SSA_WARPS;      // warps per block in pass 1
+constexpr int kThreads = kWarps * 32;
+constexpr int kU = SSA_U;              // row loads in flight per lane, per tensor
+constexpr int kMaxChunk = 1024;        // index entries staged per block
+
+struct DecodeParams {
+  const void* q;
+  const void* k;
+  const void* v;
+  const int32_t* ctx_lens;
+  const int32_t* index;     // sparse only
+  const int32_t* counts;    // sparse only (NULL selects the dense count)
+  void* out;
+  float* lse;
+  float* ws_acc;            // [B*H*n_chunks, D]
+  float2* ws_ml;            // [B*H*n_chunks]  (max in log2 units, sum)
+  uint32_t* dev_status;
+  int64_t q_sb, q_sh, k_sb, k_st, k_sh, v_sb, v_st, v_sh, o_sb, o_sh;
+  int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32;
+  float scale_log2;         // softmax scale * log2(e)
+};
+
+// Number of list entries (dense: positions) of request b, clamped to what the
+// host sized the launch for.
+__device__ __forceinline__ void request_sizes(const DecodeParams& p, int b, int& n, int& c,
+                                              uint32_t& flags) {
+  n = p.ctx_lens[b];
+  if (n > p.max_ctx) { n = p.max_ctx; flags |= SSA_DEV_BAD_COUNT; }
+  if (n < 0) n = 0;
+  if (p.counts) {
+    c = p.counts[b];
+    if (c > p.max_selected) { c = p.max_selected; flags |= SSA_DEV_BAD_COUNT; }
+    if (c < 0) c = 0;
+  } else {
+    c = n;
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void store_out(const DecodeParams& p, int b, int h, int d, float val) {
+  const int64_t o = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
+  if (p.out_f32) reinterpret_cast<float*>(p.out)[o] = val;
+  else reinterpret_cast<T*>(p.out)[o] = from_float<T>(val);
+}
+
+template <typename T, int D, bool kSparse>
+__global__ void __launch_bounds__(kThreads)
+decode_partial_kernel(const DecodeParams p) {
+  constexpr int kLanesPerRow = D / 8;                 // 16-byte pieces per row
+  constexpr int kRowsPerLoad = 32 / kLanesPerRow;     // rows one warp-wide load covers
+  constexpr int kTileRows = kRowsPerLoad * kU;        // rows per warp per iteration
+  constexpr int kGroups = kWarps * kRowsPerLoad;      // independent softmax streams
+  static_assert(kThreads >= D, "the epilogue uses one thread per output element");
+
+  __shared__ int32_t s_idx[kSparse ? kMaxChunk : 1];
+  __shared__ __align__(16) float s_acc[kGroups][D];
+  __shared__ float s_m[kGroups], s_l[kGroups];
+
+  const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int col = lane % kLanesPerRow, sub = lane / kLanesPerRow;
+
+  uint32_t flags = 0;
+  int n, c;
+  request_sizes(p, b, n, c, flags);
+  const int start = chunk_id * p.chunk;
+  if (start >= c && chunk_id > 0) return;             // chunk 0 always reports
+  const int cnt = max(0, min(p.chunk, c - start));
+
+  if (kSparse) {
+    const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
+    for (int i = tid; i < cnt; i += kThreads) {
+      int v = row[i];
+      if (v < 0 || v >= n) { v = -1; flags |= SSA_DEV_BAD_INDEX; }
+      s_idx[i] = v;
+    }
+  }
+  if (p.dev_status && h == 0) {
+    const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
+    if (f) atomicOr(p.dev_status, f);
+  }
+
+  float qf[8];
+  {
+    const T* qp = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + col * 8;
+    unpack8<T>(*reinterpret_cast<const uint4*>(qp), qf);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qf[i] *= p.scale_log2;
+  }
+  if (kSparse) __syncthreads();
+
+  const T* kbase = reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)h * p.k_sh + col * 8;
+  const T* vbase = reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)h * p.v_sh + col * 8;
+
+  float m = neg_inf(), l = 0.f;
+  float acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+
+  for (int t = warp * kTileRows; t < cnt; t += kWarps * kTileRows) {
+    uint4 kr[kU], vr[kU];
+    bool ok[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const int r = t + u * kRowsPerLoad + sub;
+      int pos = -1;
+      if (r < cnt) pos = kSparse ? s_idx[r] : start + r;
+      ok[u] = pos >= 0;
+      if (ok[u]) {
+        kr[u] = ld_stream_16B(kbase + (int64_t)pos * p.k_st);
+        vr[u] = ld_stream_16B(vbase + (int64_t)pos * p.v_st);
+      } else {
+        kr[u] = make_uint4(0, 0, 0, 0);
+        vr[u] = make_uint4(0, 0, 0, 0);
+      }
+    }
+    float s[kU];
+    float mt = neg_inf();
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      float kf[8];
+      unpack8<T>(kr[u], kf);
+      float d = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) d = fmaf(qf[i], kf[i], d);
+#pragma unroll
+      for (int o = kLanesPerRow / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      s[u] = ok[u] ? d : neg_inf();
+      mt = fmaxf(mt, s[u]);
+    }
+    const float m_new = fmaxf(m, mt);
+    if (m_new > neg_inf()) {
+      const float alpha = fast_exp2(m - m_new);       // m = -inf gives 0
+      l *= alpha;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] *= alpha;
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+        const float pw = fast_exp2(s[u] - m_new);     // masked rows give 0
+        l += pw;
+        float vf[8];
+        unpack8<T>(vr[u], vf);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw, vf[i], acc[i]);
+      }
+      m = m_new;
+    }
+  }
+
+  // combine the lane groups of the block
+  const int g = warp * kRowsPerLoad + sub;
+  *reinterpret_cast<float4*>(&s_acc[g][col * 8]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+  *reinterpret_cast<float4*>(&s_acc[g][col * 8 + 4]) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  if (col == 0) { s_m[g] = m; s_l[g] = l; }
+  __syncthreads();
+  if (tid < D) {
+    float M = neg_inf();
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i) M = fmaxf(M, s_m[i]);
+    float L = 0.f, A = 0.f;
+#pragma unroll
+    for (int i = 0; i < kGroups; ++i) {
+      const float w = (s_m[i] > neg_inf()) ? fast_exp2(s_m[i] - M) : 0.f;
+      L = fmaf(s_l[i], w, L);
+      A = fmaf(s_acc[i][tid], w, A);
+    }
+    if (p.n_chunks == 1) {
+      store_out<T>(p, b, h, tid, L > 0.f ? A / L : 0.f);
+      if (tid == 0 && p.lse) p.lse[(int64_t)b * p.H + h] = L > 0.f ? (M + log2f(L)) * kLn2 : neg_inf();
+    } else {
+      const int64_t slot = ((int64_t)b * p.H + h) * p.n_chunks + chunk_id;
+      p.ws_acc[slot * D + tid] = A;
+      if (tid == 0) p.ws_ml[slot] = make_float2(M, L);
+    }
+  }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(D)
+decode_merge_kernel(const DecodeParams p) {
+  const int h = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
+  uint32_t flags = 0;
+  int n, c;
+  request_sizes(p, b, n, c, flags);
+  const int ns = c > 0 ? (c + p.chunk - 1) / p.chunk : 1;
+  const int64_t base = ((int64_t)b * p.H + h) * p.n_chunks;
+  float M = neg_inf();
+  for (int k = 0; k < ns; ++k) M = fmaxf(M, p.ws_ml[base + k].x);
+  float L = 0.f, A = 0.f;
+  for (int k = 0; k < ns; ++k) {
+    const float2 ml = p.ws_ml[base + k];
+    const float w = (ml.x > neg_inf()) ? fast_exp2(ml.x - M) : 0.f;
+    L = fmaf(ml.y, w, L);
+    A = fmaf(p.ws_acc[(base + k) * D + d], w, A);
+  }
+  store_out<T>(p, b, h, d, L > 0.f ? A / L : 0.f);
+  if (d == 0 && p.lse) p.lse[(int64_t)b * p.H + h] = L > 0.f ? (M + log2f(L)) * kLn2 : neg_inf();
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+struct Plan { int chunk, n_chunks; size_t acc_bytes, total_bytes; };
+
+static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
+  if (!d || d->B <= 0 || d->H <= 0 || max_selected <= 0) return false;
+  if (d->D != 64 && d->D != 128) return false;
+  const long long units = (long long)d->B * d->H;
+  const long long want = 148 * 8;                     // blocks for one full wave
+  int chunk = 256;
+  while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
+  int n_chunks = (max_selected + chunk - 1) / chunk;
+  if (n_chunks == 1) chunk = (max_selected + 31) / 32 * 32;
+  pl->chunk = chunk;
+  pl->n_chunks = n_chunks;
+  pl->acc_bytes = ((size_t)units * n_chunks * d->D * sizeof(float) + 255) / 256 * 256;
+  pl->total_bytes = pl->acc_bytes + ((size_t)units * n_chunks * sizeof(float2) + 255) / 256 * 256;
+  return true;
+}
+
+static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+static int32_t check_desc(const ssa_attn_desc* d) {
+  if (d->B <= 0 || d->H <= 0 || d->max_ctx <= 0 || d->B > 65535 || d->H > 65535) return SSA_ERR_SHAPE;
+  if (d->D != 64 && d->D != 128) return SSA_ERR_UNSUPPORTED;
+  if (d->H_kv != d->H) return SSA_ERR_UNSUPPORTED;
+  if (d->kv_dtype != SSA_F16 && d->kv_dtype != SSA_BF16) return SSA_ERR_DTYPE;
+  if (d->out_dtype != d->kv_dtype && d->out_dtype != SSA_F32) return SSA_ERR_DTYPE;
+  const int64_t strides[] = {d->q_stride_b, d->q_stride_h, d->k_stride_b, d->k_stride_t, d->k_stride_h,
+                             d->v_stride_b, d->v_stride_t, d->v_stride_h, d->o_stride_b, d->o_stride_h};
+  for (int64_t s : strides) {
+    if (s < 0) return SSA_ERR_SHAPE;
+    if (s % 8 != 0) return SSA_ERR_ALIGN;
+  }
+  return SSA_OK;
+}
+
+template <typename T, int D>
+static int32_t launch(const DecodeParams& p, int B, bool sparse, cudaStream_t st) {
+  cudaEvent_t ev_b, ev_e;
+  take_kernel_events(&ev_b, &ev_e);
+  dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
+  if (ev_b) cudaEventRecord(ev_b, st);
+  if (sparse) decode_partial_kernel<T, D, true><<<grid, kThreads, 0, st>>>(p);
+  else decode_partial_kernel<T, D, false><<<grid, kThreads, 0, st>>>(p);
+  if (ev_e) cudaEventRecord(ev_e, st);
+  if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  int launches = 1;
+  if (p.n_chunks > 1) {
+    decode_merge_kernel<T, D><<<dim3((unsigned)p.H, (unsigned)B), D, 0, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+    ++launches;
+  }
+  note_launches(launches);
+  return SSA_OK;
+}
+
+static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const void* v,
+                   const int32_t* ctx_lens, const int32_t* index, int32_t index_stride,
+                   const int32_t* counts, int32_t max_selected, void* out, float* lse,
+                   void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream, bool sparse) {
+  if (!d || !q || !k || !v || !ctx_lens || !out) return SSA_ERR_NULL;
+  if (sparse && (!index || !counts)) return SSA_ERR_NULL;
+  const int32_t rc = check_desc(d);
+  if (rc != SSA_OK) return rc;
+  if (sparse) {
+    if (index_stride <= 0 || max_selected <= 0 || max_selected > index_stride) return SSA_ERR_CAPACITY;
+  } else {
+    max_selected = d->max_ctx;
+  }
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(ws)) return SSA_ERR_ALIGN;
+  Plan pl;
+  if (!make_plan(d, max_selected, &pl)) return SSA_ERR_SHAPE;
+  if (!ws || ws_bytes < pl.total_bytes) return SSA_ERR_WORKSPACE;
+
+  DecodeParams p;
+  p.q = q; p.k = k; p.v = v;
+  p.ctx_lens = ctx_lens;
+  p.index = sparse ? index : nullptr;
+  p.counts = sparse ? counts : nullptr;
+  p.out = out; p.lse = lse;
+  p.ws_acc = reinterpret_cast<float*>(ws);
+  p.ws_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(ws) + pl.acc_bytes);
+  p.dev_status = dev_status;
+  p.q_sb = d->q_stride_b; p.q_sh = d->q_stride_h;
+  p.k_sb = d->k_stride_b; p.k_st = d->k_stride_t; p.k_sh = d->k_stride_h;
+  p.v_sb = d->v_stride_b; p.v_st = d->v_stride_t; p.v_sh = d->v_stride_h;
+  p.o_sb = d->o_stride_b; p.o_sh = d->o_stride_h;
+  p.H = d->H; p.max_ctx = d->max_ctx;
+  p.index_stride = index_stride; p.max_selected = max_selected;
+  p.chunk = pl.chunk; p.n_chunks = pl.n_chunks;
+  p.out_f32 = d->out_dtype == SSA_F32;
+  const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->D);
+  p.scale_log2 = scale * kLog2e;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d->kv_dtype == SSA_BF16)
+    return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, sparse, st) : launch<__nv_bfloat16, 64>(p, d->B, sparse, st);
+  return d->D == 128 ? launch<__half, 128>(p, d->B, sparse, st) : launch<__half, 64>(p, d->B, sparse, st);
+}
+
+}  // namespace ssa
+
+extern "C" {
+
+size_t ssa_decode_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selected) {
+  ssa::Plan pl;
+  if (!desc || ssa::check_desc(desc) != SSA_OK || !ssa::make_plan(desc, max_selected, &pl)) return 0;
+  return pl.total_bytes;
+}
+
+int32_t ssa_decode_attn_sparse(const ssa_attn_desc* desc, const void* q, const void* k_cache,
+                               const void* v_cache, const int32_t* ctx_lens, const int32_t* index,
+                               int32_t index_stride, const int32_t* counts, int32_t max_selected,
+                               void* out, float* lse, void* workspace, size_t workspace_bytes,
+                               uint32_t* dev_status, void* stream) {
+  return ssa::run(desc, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out,
+                  lse, workspace, workspace_bytes, dev_status, stream, true);
+}
+
+int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q, const void* k_cache,
+                              const void* v_cache, const int32_t* ctx_lens, void* out, float* lse,
+                              void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                              void* stream) {
+  return ssa::run(desc, q, k_cache, v_cache, ctx_lens, nullptr, 0, nullptr, 0, out, lse, workspace,
+                  workspace_bytes, dev_status, stream, false);
+}
+
+}  // extern "C"

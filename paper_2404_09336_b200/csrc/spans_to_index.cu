@@ -1,0 +1,149 @@
+// Span list -> sorted duplicate-free KV index list (ssa_spans_to_index).
+//
+// One thread block per (output slice, request).  The block
+//   1. loads the request's spans, clamps them to [0, ctx_len) and packs each
+//      non-empty one into a 64-bit key (start << 32 | end);
+//   2. sorts the keys (bitonic network in shared memory);
+//   3. has one warp walk the sorted spans 32 at a time with two shuffle
+//      scans: a running maximum of the span ends seen so far, which trims
+//      each span to the part no earlier span covers, and a prefix sum of the
+//      trimmed lengths, which gives every span its offset in the output;
+//   4. writes its slice of the output: slot k finds its span by binary
+//      search over the offsets, so the stores are coalesced and balanced
+//      however uneven the spans are.
+// Blocks of one request repeat steps 1-3 (a few microseconds) instead of
+// communicating.
+#include "ssa_common.cuh"
+
+namespace ssa {
+
+constexpr int kIdxThreads = 256;
+constexpr int kMaxSpans = SSA_MAX_SPANS_PER_SEQ;   // power of two
+constexpr unsigned long long kEmptyKey = 0xffffffffffffffffull;
+
+__global__ void __launch_bounds__(kIdxThreads)
+spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* __restrict__ spans,
+                      const int32_t* __restrict__ ctx_lens, int32_t* __restrict__ index,
+                      int32_t index_stride, int32_t slice, int32_t* __restrict__ counts,
+                      uint32_t* __restrict__ dev_status) {
+  __shared__ unsigned long long keys[kMaxSpans];
+  __shared__ int32_t new_start[kMaxSpans];
+  __shared__ int32_t offs[kMaxSpans + 1];
+  __shared__ uint32_t s_flags;
+
+  const int b = blockIdx.y;
+  const int tid = threadIdx.x;
+  const int n = max(ctx_lens[b], 0);
+  const int first = span_offsets[b];
+  int S = span_offsets[b + 1] - first;
+  uint32_t flags = 0;
+  if (S < 0) S = 0;
+  if (S > kMaxSpans) { S = kMaxSpans; flags |= SSA_DEV_TOO_MANY_SPANS; }
+  int P = 32;
+  while (P < S) P <<= 1;
+  if (tid == 0) s_flags = 0;
+
+  // 1. load, clamp, pack
+  for (int i = tid; i < P; i += kIdxThreads) {
+    unsigned long long key = kEmptyKey;
+    if (i < S) {
+      const int2 se = reinterpret_cast<const int2*>(spans)[first + i];
+      if (se.x < 0 || se.x > se.y) flags |= SSA_DEV_BAD_SPAN;
+      if (se.y > n) flags |= SSA_DEV_CLIPPED;
+      const int s = max(se.x, 0), e = min(se.y, n);
+      if (e > s) key = ((unsigned long long)(uint32_t)s << 32) | (uint32_t)e;
+    }
+    keys[i] = key;
+  }
+  __syncthreads();
+
+  // 2. bitonic sort, ascending by (start, end); empty keys sink to the end
+  for (int k = 2; k <= P; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < P; i += kIdxThreads) {
+        const int ixj = i ^ j;
+        if (ixj > i) {
+          const unsigned long long a = keys[i], c = keys[ixj];
+          const bool up = (i & k) == 0;
+          if ((a > c) == up) { keys[i] = c; keys[ixj] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+
+  // 3. trim against the running maximum end and prefix-sum the lengths
+  if (tid < 32) {
+    int run_max = 0, run_sum = 0;
+    for (int base = 0; base < P; base += 32) {
+      const unsigned long long key = keys[base + tid];
+      const bool live = key != kEmptyKey;
+      const int s = live ? (int)(key >> 32) : 0;
+      const int e = live ? (int)(uint32_t)key : 0;
+      int mx = e;                                   // inclusive max-scan of ends
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, mx, d);
+        if (tid >= d) mx = max(mx, o);
+      }
+      int prev = __shfl_up_sync(0xffffffffu, mx, 1);
+      prev = (tid == 0) ? run_max : max(prev, run_max);
+      const int ns = max(s, prev);
+      const int len = live ? max(e - ns, 0) : 0;
+      int sum = len;                                // inclusive sum-scan of lengths
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, sum, d);
+        if (tid >= d) sum += o;
+      }
+      new_start[base + tid] = ns;
+      offs[base + tid] = run_sum + sum - len;
+      run_max = max(run_max, __shfl_sync(0xffffffffu, mx, 31));
+      run_sum += __shfl_sync(0xffffffffu, sum, 31);
+    }
+    if (tid == 0) offs[P] = run_sum;
+  }
+  if (flags) atomicOr(&s_flags, flags);
+  __syncthreads();
+
+  const int total = offs[P];
+  const int c = min(total, index_stride);
+  if (blockIdx.x == 0 && tid == 0) {
+    counts[b] = c;
+    uint32_t f = s_flags;
+    if (total > index_stride) f |= SSA_DEV_OVERFLOW;
+    if (f && dev_status) atomicOr(dev_status, f);
+  }
+
+  // 4. write this block's slice of the list
+  const int k_end = min(c, (int)(blockIdx.x + 1) * slice);
+  int32_t* row = index + (size_t)b * index_stride;
+  for (int k = blockIdx.x * slice + tid; k < k_end; k += kIdxThreads) {
+    int lo = 0, hi = P;                             // last i with offs[i] <= k
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (offs[mid] <= k) lo = mid; else hi = mid;
+    }
+    row[k] = new_start[lo] + (k - offs[lo]);
+  }
+}
+
+}  // namespace ssa
+
+extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t* spans,
+                                      const int32_t* ctx_lens, int32_t B, int32_t* index,
+                                      int32_t index_stride, int32_t* counts,
+                                      uint32_t* dev_status, void* stream) {
+  if (!span_offsets || !spans || !ctx_lens || !index || !counts) return SSA_ERR_NULL;
+  if (B <= 0 || B > 65535 || index_stride <= 0) return SSA_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(spans) % 8 != 0) return SSA_ERR_ALIGN;
+  int slices = (index_stride + 2047) / 2048;
+  if (slices > 8) slices = 8;
+  const int32_t slice = (index_stride + slices - 1) / slices;
+  dim3 grid((unsigned)slices, (unsigned)B);
+  ssa::spans_to_index_kernel<<<grid, ssa::kIdxThreads, 0, (cudaStream_t)stream>>>(
+      span_offsets, spans, ctx_lens, index, index_stride, slice, counts, dev_status);
+  if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  ssa::note_launches(1);
+  return SSA_OK;
+}

@@ -1,0 +1,158 @@
+"""ctypes binding of libssa (include/ssa.h): argument marshalling only.
+
+Every function takes torch CUDA tensors (used purely as device memory) and
+hands their addresses, sizes and strides to the C entry point of the same
+name.  Nothing is computed here, and there is no fallback: if the shared
+library cannot be loaded the import fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+# ---- status codes / bits (mirror include/ssa.h) -----------------------------------
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED = range(1, 9)
+DEV_BAD_SPAN, DEV_CLIPPED, DEV_OVERFLOW, DEV_BAD_INDEX, DEV_BAD_COUNT, DEV_TOO_MANY_SPANS = 1, 2, 4, 8, 16, 32
+MAX_SPANS_PER_SEQ = 2048
+F16, BF16, F32 = 0, 1, 2
+_DTYPES = {torch.float16: F16, torch.bfloat16: BF16, torch.float32: F32}
+
+
+class AttnDesc(C.Structure):
+    _fields_ = [
+        ("B", C.c_int32), ("H", C.c_int32), ("H_kv", C.c_int32), ("D", C.c_int32),
+        ("max_ctx", C.c_int32), ("kv_dtype", C.c_int32), ("out_dtype", C.c_int32), ("scale", C.c_float),
+        ("q_stride_b", C.c_int64), ("q_stride_h", C.c_int64),
+        ("k_stride_b", C.c_int64), ("k_stride_t", C.c_int64), ("k_stride_h", C.c_int64),
+        ("v_stride_b", C.c_int64), ("v_stride_t", C.c_int64), ("v_stride_h", C.c_int64),
+        ("o_stride_b", C.c_int64), ("o_stride_h", C.c_int64),
+    ]
+
+
+class SsaError(RuntimeError):
+    def __init__(self, fn, code):
+        self.code = code
+        super().__init__(f"{fn}: {status_string(code)} (status {code})")
+
+
+def _load():
+    path = os.environ.get("SSA_LIBRARY") or _build.LIB
+    if path == _build.LIB:
+        _build.build_library()          # no-op when the in-tree library is current
+    lib = C.CDLL(path)
+    vp = C.c_void_p
+    lib.ssa_spans_to_index.restype = C.c_int32
+    lib.ssa_spans_to_index.argtypes = [vp, vp, vp, C.c_int32, vp, C.c_int32, vp, vp, vp]
+    lib.ssa_decode_workspace_bytes.restype = C.c_size_t
+    lib.ssa_decode_workspace_bytes.argtypes = [C.POINTER(AttnDesc), C.c_int32]
+    lib.ssa_decode_attn_sparse.restype = C.c_int32
+    lib.ssa_decode_attn_sparse.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
+                                           vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_attn_dense.restype = C.c_int32
+    lib.ssa_decode_attn_dense.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_set_kernel_events.restype = None
+    lib.ssa_set_kernel_events.argtypes = [vp, vp]
+    lib.ssa_launch_count.restype = C.c_uint64
+    lib.ssa_launch_count.argtypes = []
+    lib.ssa_status_string.restype = C.c_char_p
+    lib.ssa_status_string.argtypes = [C.c_int32]
+    lib.ssa_version.restype = C.c_int32
+    lib.ssa_version.argtypes = []
+    return lib
+
+
+lib = _load()
+LIBRARY_PATH = lib._name
+
+
+def status_string(code: int) -> str:
+    return lib.ssa_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return lib.ssa_version()
+
+
+def launch_count() -> int:
+    return int(lib.ssa_launch_count())
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(fn, rc, check):
+    if check and rc != OK:
+        raise SsaError(fn, rc)
+    return rc
+
+
+def make_desc(q, k_cache, v_cache, out, max_ctx=None, scale: float = 0.0) -> AttnDesc:
+    """Descriptor for q[B,H,D], k_cache/v_cache[B,H,T,D] (any batch, head and
+    token strides: a token-major cache is the permuted view) and out[B,H,D]."""
+    B, H, D = q.shape
+    d = AttnDesc()
+    d.B, d.H, d.H_kv, d.D = B, H, k_cache.shape[1], D
+    d.max_ctx = int(k_cache.shape[2] if max_ctx is None else max_ctx)
+    d.kv_dtype = _DTYPES.get(k_cache.dtype, -1)
+    d.out_dtype = _DTYPES.get(out.dtype, -1)
+    d.scale = float(scale)
+    d.q_stride_b, d.q_stride_h = q.stride(0), q.stride(1)
+    d.k_stride_b, d.k_stride_h, d.k_stride_t = k_cache.stride(0), k_cache.stride(1), k_cache.stride(2)
+    d.v_stride_b, d.v_stride_h, d.v_stride_t = v_cache.stride(0), v_cache.stride(1), v_cache.stride(2)
+    d.o_stride_b, d.o_stride_h = out.stride(0), out.stride(1)
+    for t in (q, k_cache, v_cache, out):
+        if t.stride(-1) != 1:
+            raise ValueError("the head dimension must be contiguous")
+    return d
+
+
+def spans_to_index(span_offsets, spans, ctx_lens, index, counts, dev_status=None, stream=None, check=True):
+    """ssa_spans_to_index: index[B, index_stride] and counts[B] are written."""
+    rc = lib.ssa_spans_to_index(_ptr(span_offsets), _ptr(spans), _ptr(ctx_lens), int(ctx_lens.numel()),
+                                _ptr(index), int(index.stride(0)), _ptr(counts), _ptr(dev_status),
+                                _stream(stream))
+    return _check("ssa_spans_to_index", rc, check)
+
+
+def decode_workspace_bytes(desc: AttnDesc, max_selected: int) -> int:
+    return int(lib.ssa_decode_workspace_bytes(C.byref(desc), int(max_selected)))
+
+
+def decode_attn_sparse(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_selected, out, lse=None,
+                       workspace=None, dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_sparse: out (and lse) are written."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_sparse(C.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens),
+                                    _ptr(index), int(index.stride(0)) if index is not None else 0,
+                                    _ptr(counts), int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace),
+                                    ws_bytes, _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_sparse", rc, check)
+
+
+def decode_attn_dense(desc, q, k_cache, v_cache, ctx_lens, out, lse=None, workspace=None, dev_status=None,
+                      stream=None, check=True):
+    """ssa_decode_attn_dense: out (and lse) are written."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_dense(C.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens),
+                                   _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes, _ptr(dev_status),
+                                   _stream(stream))
+    return _check("ssa_decode_attn_dense", rc, check)
+
+
+def set_kernel_events(begin=None, end=None):
+    """ssa_set_kernel_events with torch.cuda.Event objects that have been
+    recorded at least once (so that they own a CUDA event), or None."""
+    lib.ssa_set_kernel_events(None if begin is None else C.c_void_p(begin.cuda_event),
+                              None if end is None else C.c_void_p(end.cuda_event))

@@ -1,0 +1,114 @@
+"""The C-ABI library loads, exports what include/ssa.h declares, and rejects
+bad arguments on the host before anything is launched (no GPU needed)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2404_09336_b200 import ssa
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ssa.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ssa_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_symbols()
+    assert {"ssa_spans_to_index", "ssa_decode_attn_sparse", "ssa_decode_attn_dense",
+            "ssa_decode_workspace_bytes"} <= set(names)
+    raw = C.CDLL(ssa.LIBRARY_PATH)
+    for n in names:
+        assert hasattr(raw, n), n
+
+
+def test_library_is_in_tree():
+    assert os.path.dirname(ssa.LIBRARY_PATH) == os.path.join(ROOT, "paper_2404_09336_b200")
+
+
+def test_version_and_strings():
+    assert ssa.version() >= 100
+    assert ssa.status_string(ssa.OK) == "ok"
+    assert "aligned" in ssa.status_string(ssa.ERR_ALIGN)
+    assert "unknown" in ssa.status_string(12345)
+
+
+def good_desc():
+    d = ssa.AttnDesc()
+    d.B, d.H, d.H_kv, d.D, d.max_ctx = 2, 4, 4, 128, 512
+    d.kv_dtype, d.out_dtype, d.scale = ssa.BF16, ssa.BF16, 0.0
+    d.q_stride_b, d.q_stride_h = 4 * 128, 128
+    d.k_stride_b, d.k_stride_h, d.k_stride_t = 4 * 512 * 128, 512 * 128, 128
+    d.v_stride_b, d.v_stride_h, d.v_stride_t = 4 * 512 * 128, 512 * 128, 128
+    d.o_stride_b, d.o_stride_h = 4 * 128, 128
+    return d
+
+
+def test_workspace_query():
+    d = good_desc()
+    small = ssa.decode_workspace_bytes(d, 64)
+    full = ssa.decode_workspace_bytes(d, 512)
+    assert 0 < small <= full
+    assert full >= 2 * 4 * (512 // 256) * (128 * 4 + 8)
+    d.D = 96
+    assert ssa.decode_workspace_bytes(d, 64) == 0
+    d = good_desc()
+    assert ssa.decode_workspace_bytes(d, 0) == 0
+
+
+P = C.c_void_p(0x1000)      # never dereferenced: validation fails first
+NUL = None
+
+
+def sparse(d, q=P, k=P, v=P, ctx=P, idx=P, stride=64, cnt=P, max_sel=64, out=P, ws=P, ws_bytes=1 << 30):
+    return ssa.lib.ssa_decode_attn_sparse(C.byref(d), q, k, v, ctx, idx, stride, cnt, max_sel, out, NUL, ws,
+                                          ws_bytes, NUL, NUL)
+
+
+def test_sparse_rejects_bad_arguments_without_launching():
+    before = ssa.launch_count()
+    d = good_desc()
+    assert ssa.lib.ssa_decode_attn_sparse(None, P, P, P, P, P, 64, P, 64, P, NUL, P, 1 << 30, NUL, NUL) == ssa.ERR_NULL
+    assert sparse(d, q=NUL) == ssa.ERR_NULL
+    assert sparse(d, idx=NUL) == ssa.ERR_NULL
+    assert sparse(d, out=NUL) == ssa.ERR_NULL
+    assert sparse(d, max_sel=65) == ssa.ERR_CAPACITY
+    assert sparse(d, max_sel=0) == ssa.ERR_CAPACITY
+    assert sparse(d, stride=0) == ssa.ERR_CAPACITY
+    assert sparse(d, k=C.c_void_p(0x1008)) == ssa.ERR_ALIGN
+    assert sparse(d, ws=NUL) == ssa.ERR_WORKSPACE
+    assert sparse(d, ws_bytes=16) == ssa.ERR_WORKSPACE
+    for field, val, err in [("D", 96, ssa.ERR_UNSUPPORTED), ("H_kv", 2, ssa.ERR_UNSUPPORTED),
+                            ("kv_dtype", ssa.F32, ssa.ERR_DTYPE), ("out_dtype", ssa.F16, ssa.ERR_DTYPE),
+                            ("k_stride_t", 132, ssa.ERR_ALIGN), ("B", 0, ssa.ERR_SHAPE),
+                            ("max_ctx", 0, ssa.ERR_SHAPE), ("v_stride_h", -128, ssa.ERR_SHAPE)]:
+        d = good_desc()
+        setattr(d, field, val)
+        assert sparse(d) == err, field
+    assert ssa.launch_count() == before
+
+
+def test_dense_and_index_reject_bad_arguments():
+    before = ssa.launch_count()
+    d = good_desc()
+    f = ssa.lib.ssa_decode_attn_dense
+    assert f(C.byref(d), P, P, P, NUL, P, NUL, P, 1 << 30, NUL, NUL) == ssa.ERR_NULL
+    assert f(C.byref(d), P, P, P, P, P, NUL, P, 64, NUL, NUL) == ssa.ERR_WORKSPACE
+    d.D = 32
+    assert f(C.byref(d), P, P, P, P, P, NUL, P, 1 << 30, NUL, NUL) == ssa.ERR_UNSUPPORTED
+    g = ssa.lib.ssa_spans_to_index
+    assert g(NUL, P, P, 4, P, 64, P, NUL, NUL) == ssa.ERR_NULL
+    assert g(P, P, P, 0, P, 64, P, NUL, NUL) == ssa.ERR_SHAPE
+    assert g(P, P, P, 4, P, 0, P, NUL, NUL) == ssa.ERR_SHAPE
+    assert g(P, C.c_void_p(0x1004), P, 4, P, 64, P, NUL, NUL) == ssa.ERR_ALIGN
+    assert ssa.launch_count() == before
+
+
+def test_error_raises_through_binding():
+    with pytest.raises(ssa.SsaError) as e:
+        ssa._check("ssa_decode_attn_sparse", ssa.ERR_WORKSPACE, True)
+    assert "workspace" in str(e.value)
