@@ -41,7 +41,11 @@ def round_to_storage(x32: np.ndarray, dtype: str) -> np.ndarray:
         return x32.astype(np.float16).view(np.uint16)
     if dtype == "bf16":
         u = x32.view(np.uint32)
-        return ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+        t = u >> np.uint32(16)              # u + 0x7FFF + (bit 16 of u), then keep the upper half
+        t &= np.uint32(1)
+        t += np.uint32(0x7FFF)
+        t += u
+        return (t >> np.uint32(16)).astype(np.uint16)
     raise ValueError(dtype)
 
 

@@ -1,0 +1,238 @@
+"""ssa_decode_attn_sparse / ssa_decode_attn_dense against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssa_oracle as O
+from paper_2404_09336_b200 import inputs, ssa
+from paper_2404_09336_b200.runner import DecodeStep
+
+from gpu_util import Problem
+from parity import assert_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def scale_of(D):
+    return 1.0 / np.sqrt(D)
+
+
+def oracle_for(wl, ds, seqs=None, heads=None):
+    """Oracle output for a workload from the generator's own bits (never from
+    device memory): index lists by the oracle, attention in set form."""
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, ds.index_stride)
+    seqs = list(range(wl.B)) if seqs is None else list(seqs)
+    q = wl.q_bits()
+    out = np.full((wl.B, wl.H, wl.D), np.nan)
+    lse = np.full((wl.B, wl.H), np.nan)
+    dense = np.full((wl.B, wl.H, wl.D), np.nan)
+    for b in seqs:
+        k, v = wl.kv_bits_seq(b)
+        o, l = O.decode_attn_sparse(q[b:b + 1], k[None], v[None], wl.ctx_lens[b:b + 1], index[b:b + 1],
+                                    counts[b:b + 1], scale_of(wl.D), wl.dtype, heads=heads)
+        out[b], lse[b] = o[0], l[0]
+        od, _ = O.decode_attn_dense(q[b:b + 1], k[None], v[None], wl.ctx_lens[b:b + 1], scale_of(wl.D),
+                                    wl.dtype, heads=heads)
+        dense[b] = od[0]
+    return out, lse, dense, index, counts
+
+
+def run_and_compare(wl, layout="bhtd", out_dtype=None, seqs=None, heads=None):
+    ds = DecodeStep(wl, layout=layout, out_dtype=out_dtype)
+    ref, ref_lse, ref_dense, ref_index, ref_counts = oracle_for(wl, ds, seqs, heads)
+    ds.step()
+    torch.cuda.synchronize()
+    assert int(ds.status.item()) == 0
+    counts = ds.counts.cpu().numpy()
+    assert counts.tolist() == ref_counts.tolist()
+    idx = ds.index.cpu().numpy()
+    for b in range(wl.B):
+        assert np.array_equal(idx[b, :counts[b]], ref_index[b, :counts[b]])
+    got, got_lse = ds.out_f64(), ds.lse.double().cpu().numpy()
+    native = out_dtype is None
+    sel = ~np.isnan(ref)
+    r = assert_parity(got[sel], ref[sel], native, f"{wl.name} sparse {layout}")
+    sel_l = ~np.isnan(ref_lse)
+    np.testing.assert_allclose(got_lse[sel_l], ref_lse[sel_l], rtol=1e-5, atol=1e-5)
+    ds.out.fill_(55.0)
+    ds.attend_dense()
+    torch.cuda.synchronize()
+    assert int(ds.status.item()) == 0
+    assert_parity(ds.out_f64()[sel], ref_dense[sel], native, f"{wl.name} dense {layout}")
+    return r
+
+
+# ---- the five workloads, scaled so that the oracle covers every output ----------------
+@pytest.mark.parametrize("layout", ["bhtd", "bthd"])
+@pytest.mark.parametrize("out_dtype", [None, torch.float32])
+def test_cfg1_tiny_full(layout, out_dtype):
+    run_and_compare(inputs.make_config(1), layout, out_dtype)
+
+
+@pytest.mark.parametrize("layout", ["bhtd", "bthd"])
+@pytest.mark.parametrize("out_dtype", [None, torch.float32])
+def test_cfg2_reduced(layout, out_dtype):
+    run_and_compare(inputs.make_config(2, B=6, H=4), layout, out_dtype)
+
+
+@pytest.mark.parametrize("out_dtype", [None, torch.float32])
+def test_cfg3_reduced(out_dtype):
+    run_and_compare(inputs.make_config(3, B=3, H=3), "bhtd", out_dtype)
+
+
+def test_cfg4_reduced():
+    run_and_compare(inputs.make_config(4, B=2, H=2), "bhtd", torch.float32)
+    run_and_compare(inputs.make_config(4, B=1, H=2), "bthd", None)
+
+
+@pytest.mark.parametrize("f", [0.01, 0.10, 1.00])
+def test_cfg5_reduced(f):
+    run_and_compare(inputs.make_config(5, density=f, B=2, H=2), "bhtd", torch.float32)
+
+
+# ---- full sizes, in the launch configuration the benchmark times; sampled outputs -----
+@pytest.mark.parametrize("cfg,density", [(2, None), (3, None), (4, None), (5, 0.05), (5, 0.50)])
+def test_full_size_sampled(cfg, density):
+    wl = inputs.make_config(cfg, density=density)
+    rng = np.random.default_rng(cfg)
+    seqs = sorted(rng.choice(wl.B, size=2, replace=False).tolist())
+    heads = sorted(rng.choice(wl.H, size=3, replace=False).tolist())
+    run_and_compare(wl, "bhtd", None, seqs=seqs, heads=heads)
+
+
+# ---- edge cases on hand-made problems ----------------------------------------------------
+def oracle_sparse(p, ctx, index, counts, scale=None):
+    return O.decode_attn_sparse(p.q_bits, p.k_bits, p.v_bits, ctx, index, counts,
+                                scale_of(p.D) if scale is None else scale, p.dtype)
+
+
+@pytest.mark.parametrize("dtype,D", [("bf16", 128), ("f16", 128), ("bf16", 64), ("f16", 64)])
+@pytest.mark.parametrize("layout", ["bhtd", "bthd"])
+def test_counts_zero_one_and_ragged(dtype, D, layout):
+    B, H, T = 5, 3, 700
+    p = Problem(B, H, T, D, dtype, seed=D, layout=layout)
+    ctx = [700, 1, 513, 64, 300]
+    rng = np.random.default_rng(0)
+    index = np.full((B, 704), -1, np.int32)
+    counts = [0, 1, 513, 17, 300]
+    index[1, 0] = 0
+    index[2, :513] = np.arange(513)
+    index[3, :17] = np.sort(rng.choice(64, 17, replace=False))
+    index[4, :300] = rng.permutation(300)                     # unsorted list
+    for out_dtype in (torch.float32, None):
+        out, lse, status, _ = p.sparse(ctx, index, counts, out_dtype=out_dtype)
+        ref, ref_lse = oracle_sparse(p, ctx, index, counts)
+        assert status == 0
+        assert not out[0].any() and np.all(np.isneginf(lse[0]))            # empty selection
+        assert_parity(out, ref, out_dtype is None, "edge")
+        np.testing.assert_allclose(lse[1:], ref_lse[1:], rtol=1e-5, atol=1e-5)
+    # a single selected row is returned exactly
+    out, _, _, _ = p.sparse(ctx, index, counts, out_dtype=torch.float32)
+    assert np.array_equal(out[1], O.decode_bits(p.v_bits[1, :, 0, :], dtype))
+
+
+def test_multi_chunk_merge_and_tail_sizes():
+    # sizes around the tile, chunk and split boundaries
+    B, H, T, D = 1, 2, 3000, 128
+    p = Problem(B, H, T, D, "bf16", seed=7)
+    rng = np.random.default_rng(3)
+    for c in (1, 15, 16, 17, 63, 64, 65, 255, 256, 257, 511, 513, 1000, 2999, 3000):
+        index = np.full((B, 3008), -1, np.int32)
+        index[0, :c] = np.sort(rng.choice(T, c, replace=False))
+        for ms in {c, 3000}:
+            out, lse, status, _ = p.sparse([T], index, [c], max_selected=ms)
+            ref, ref_lse = oracle_sparse(p, [T], index, [c])
+            assert status == 0
+            assert_parity(out, ref, False, f"c={c} ms={ms}")
+            np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+
+
+def test_full_span_equals_dense():
+    B, H, T, D = 3, 2, 1500, 128
+    p = Problem(B, H, T, D, "bf16", seed=11)
+    ctx = [1500, 777, 1]
+    index = np.tile(np.arange(1504, dtype=np.int32), (B, 1))
+    out_s, lse_s, st, _ = p.sparse(ctx, index, ctx, max_selected=1500)
+    out_d, lse_d, st_d = p.dense(ctx)
+    ref, ref_lse = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, ctx, scale_of(D), "bf16")
+    assert st == 0 and st_d == 0
+    assert_parity(out_s, ref, False, "sparse full span")
+    assert_parity(out_d, ref, False, "dense")
+    np.testing.assert_allclose(out_s, out_d, rtol=0, atol=1e-5)
+    np.testing.assert_allclose(lse_d, ref_lse, rtol=1e-5, atol=1e-5)
+    np.testing.assert_allclose(lse_s, ref_lse, rtol=1e-5, atol=1e-5)
+
+
+def test_unselected_rows_do_not_matter():
+    B, H, T, D = 2, 2, 600, 128
+    p = Problem(B, H, T, D, "bf16", seed=13)
+    ctx = [600, 400]
+    rng = np.random.default_rng(1)
+    index = np.full((B, 608), -1, np.int32)
+    counts = [150, 90]
+    index[0, :150] = np.sort(rng.choice(600, 150, replace=False))
+    index[1, :90] = np.sort(rng.choice(400, 90, replace=False))
+    base, base_lse, _, _ = p.sparse(ctx, index, counts)
+    for b in range(B):                                         # poison everything unselected
+        keep = np.zeros(T, bool)
+        keep[index[b, :counts[b]]] = True
+        p.k_bits[b][:, ~keep, :] = 0x7FC0                      # NaN
+        p.v_bits[b][:, ~keep, :] = 0x7F80                      # +inf
+    p.upload()
+    out, lse, status, _ = p.sparse(ctx, index, counts)
+    assert status == 0
+    assert np.array_equal(out, base) and np.array_equal(lse, base_lse)
+    ref, _ = oracle_sparse(p, ctx, index, counts)
+    assert_parity(out, ref, False, "poisoned")
+
+
+def test_bad_entries_are_skipped_and_flagged():
+    B, H, T, D = 2, 2, 300, 64
+    p = Problem(B, H, T, D, "f16", seed=17)
+    ctx = [200, 300]
+    index = np.full((B, 64), -1, np.int32)
+    index[0, :6] = [5, 250, 7, -3, 199, 200]                  # 250, -3, 200 are outside [0, 200)
+    index[1, :4] = [1, 1, 2, 299]                             # a duplicate counts twice
+    counts = [6, 4]
+    out, lse, status, _ = p.sparse(ctx, index, counts)
+    assert status == ssa.DEV_BAD_INDEX
+    ref, ref_lse = oracle_sparse(p, ctx, index, counts)
+    assert_parity(out, ref, False, "bad entries")
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+    # a count above the host bound is clamped and flagged
+    index[0, :40] = np.arange(40)
+    out, _, status, _ = p.sparse(ctx, index, [40, 4], max_selected=32)
+    assert status & ssa.DEV_BAD_COUNT
+    ref, _ = oracle_sparse(p, ctx, index, [32, 4])
+    assert_parity(out, ref, False, "clamped count")
+    # a context length above the allocated rows is clamped and flagged (dense)
+    out, _, status = p.dense([999, 300])
+    assert status & ssa.DEV_BAD_COUNT
+    ref, _ = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, [300, 300], scale_of(D), "f16")
+    assert_parity(out, ref, False, "clamped ctx")
+
+
+def test_explicit_scale_and_large_scores():
+    B, H, T, D = 1, 2, 256, 128
+    p = Problem(B, H, T, D, "bf16", seed=19)
+    index = np.arange(256, dtype=np.int32)[None]
+    for scale in (1.0, 0.01):                                 # scale 1: nearly one-hot softmax
+        out, lse, _, _ = p.sparse([256], index, [256], scale=scale)
+        ref, ref_lse = oracle_sparse(p, [256], index, [256], scale=scale)
+        assert_parity(out, ref, False, f"scale {scale}")
+        np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-4)
+
+
+def test_strided_views_and_launch_counter():
+    # q and out as slices of larger buffers (strides differ from the packed ones)
+    B, H, T, D = 2, 3, 128, 128
+    p = Problem(B, H, T, D, "bf16", seed=23)
+    big_q = torch.zeros((B, H, 2 * D), dtype=torch.bfloat16, device="cuda:0")
+    big_q[:, :, :D] = p.q
+    p.q = big_q[:, :, :D]
+    index = np.tile(np.arange(0, 128, 2, dtype=np.int32), (B, 1))
+    before = ssa.launch_count()
+    out, _, status, _ = p.sparse([128, 128], index, [64, 64])
+    assert ssa.launch_count() > before
+    ref, _ = oracle_sparse(p, [128, 128], index, [64, 64])
+    assert_parity(out, ref, False, "strided q")
