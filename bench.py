@@ -1,0 +1,473 @@
+#!/usr/bin/env python
+"""Benchmark of the span-restricted decode-attention step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--cfg 2] [--sweep auto|none|all]
+
+One step = one decode step of the method over one batch: span lists -> index
+lists (ssa_spans_to_index) -> span-restricted attention
+(ssa_decode_attn_sparse).  The metric is the effective KV bandwidth: bytes of
+the selected K and V rows divided by the step time.  The dense baseline
+(ssa_decode_attn_dense) is timed beside it for the speedup.
+
+With N > 1 (torchrun, one rank per GPU) every rank runs its own batch of the
+same workload (requests are independent: no collective on the data path);
+the time is the maximum over ranks and the value the sum of all ranks' bytes.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "span-sparse decode attn: effective KV GB/s (% HBM peak); speedup vs dense"
+SPEC_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+WORKLOAD_TEXT = {
+    1: "cfg1 tiny: B=1 H=8 D=64 ctx=512 fp16",
+    2: "cfg2 arithmetic-style: B=64 H=32 D=128 ragged ctx 256-1024 bf16, prefix 64 + 1-4 spans of 4-32 + last 32",
+    3: "cfg3 summarization-style: B=16 H=32 D=128 ctx=4096 bf16",
+    4: "cfg4 long context: B=8 H=32 D=128 ctx=16384 bf16",
+    5: "cfg5 density sweep: B=32 H=32 D=128 ctx=8192 bf16",
+}
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows, self.proc, self.thread = [], None, None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, windows):
+        """windows: list of (t0, t1) wall-clock intervals in which the GPU was under load."""
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        sm, mx, reasons, n_all = [], 0.0, set(), 0
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for t, line in self.rows:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            n_all += 1
+            if not any(a <= t <= b for a, b in windows):
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx = max(mx, float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples_under_load": len(sm), "samples": n_all}
+
+
+# ---------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands
+# ---------------------------------------------------------------------------------------
+def oracle_step(O, wl, q, k, v, n_seq, stride):
+    """One decode step of the oracle over the first n_seq requests."""
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets[: n_seq + 1], wl.spans, wl.ctx_lens[:n_seq], stride)
+    out, _ = O.decode_attn_sparse(q[:n_seq], k[:n_seq], v[:n_seq], wl.ctx_lens[:n_seq], index, counts,
+                                  1.0 / math.sqrt(wl.D), wl.dtype)
+    return int(counts.sum()) * wl.kv_bytes_per_token(), out
+
+
+def time_oracle(cfg, budget_s, steps=None, warmup=0):
+    """Times the oracle on a bounded sample of workload `cfg`.  With `steps`
+    given, runs warmup + steps steps over a sample sized so that the whole run
+    takes about budget_s; otherwise repeats whole-sample steps for budget_s."""
+    from threadpoolctl import threadpool_limits
+
+    from oracle import ssa_oracle as O
+    from paper_2404_09336_b200 import inputs
+    wl = inputs.make_config(cfg)
+    stride = (wl.selected_upper_bound() + 31) // 32 * 32
+    with threadpool_limits(limits=1):
+        probe = min(wl.B, 4)
+        sub = wl.shard(0, max(wl.B // probe, 1)) if wl.B > probe else wl
+        q, (k, v) = sub.q_bits(), sub.kv_bits()
+        t0 = time.perf_counter()
+        oracle_step(O, sub, q, k, v, sub.B, stride)
+        per_seq = (time.perf_counter() - t0) / sub.B
+        if steps is None:
+            n_seq = min(wl.B, max(1, int(budget_s / 3 / per_seq)))
+        else:
+            n_seq = min(wl.B, max(1, int(budget_s / (steps + warmup) / per_seq)))
+        if n_seq > sub.B:
+            sub = wl.shard(0, 1) if n_seq == wl.B else wl.shard(0, wl.B // n_seq)
+            n_seq = min(n_seq, sub.B)
+            q, (k, v) = sub.q_bits(), sub.kv_bits()
+        for _ in range(warmup):
+            oracle_step(O, sub, q, k, v, n_seq, stride)
+        done, nbytes = 0, 0
+        t0 = time.perf_counter()
+        while True:
+            b, _ = oracle_step(O, sub, q, k, v, n_seq, stride)
+            nbytes += b
+            done += 1
+            el = time.perf_counter() - t0
+            if (steps is not None and done >= steps) or (steps is None and el >= budget_s and done >= 1):
+                break
+    return {"value": nbytes / el / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"{done} steps over the first {n_seq} of {wl.B} requests x {wl.H} heads of {WORKLOAD_TEXT[cfg].split(':')[0]} "
+                      f"({nbytes // max(done, 1)} selected KV bytes per step), numpy fp64, 1 thread",
+            "seconds": el, "ms_per_step": el / done * 1e3, "steps": done}
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    r = time_oracle(args.cfg, budget_s=90.0, steps=args.steps, warmup=args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": WORKLOAD_TEXT[args.cfg]},
+            "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------
+class Timer:
+    def __init__(self, torch, dist, world):
+        self.torch, self.dist, self.world = torch, dist, world
+        self.windows = []
+
+    def sync(self):
+        self.torch.cuda.synchronize()
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def run(self, fn, steps):
+        """Device time of `steps` calls of fn(i): events on the launching
+        stream, a barrier + synchronize on both sides, maximum over ranks."""
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.sync()
+        w0 = time.time()
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        self.sync()
+        self.windows.append((w0, time.time()))
+        ms = e0.elapsed_time(e1)
+        if self.world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def total(self, x):
+        if self.world > 1:
+            t = self.torch.tensor([float(x)], dtype=self.torch.float64, device="cuda")
+            self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM)
+            return float(t.item())
+        return float(x)
+
+
+def l2_bytes(torch):
+    return int(torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size)
+
+
+def copies_for(selected_bytes, cache_bytes, l2, cap_bytes=40e9):
+    want = max(2, math.ceil(2 * l2 / max(selected_bytes, 1)) + 1)
+    return int(max(1, min(want, 8, cap_bytes // max(cache_bytes, 1))))
+
+
+def capture_graphs(torch, ds, fn):
+    """One CUDA graph per KV copy replaying fn() (the library's launches)."""
+    graphs = []
+    side = torch.cuda.Stream()
+    for c in range(len(ds.k_store)):
+        ds.select_copy(c)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn()
+        graphs.append(g)
+    torch.cuda.synchronize()
+    return graphs
+
+
+def measure(torch, ssa, timer, ds, steps, warmup, peak, kernel_pass=True):
+    """All timings of one workload held by `ds`.  Returns a dict."""
+    ncopy = len(ds.k_store)
+
+    def rot(i):
+        ds.select_copy(i % ncopy)
+
+    for i in range(max(warmup, 3)):
+        rot(i)
+        ds.step()
+        ds.attend_dense()
+    torch.cuda.synchronize()
+    l0 = ssa.launch_count()
+    ds.step()
+    launches_per_step = ssa.launch_count() - l0
+    torch.cuda.synchronize()
+    status = int(ds.status.item())
+    sel = ds.selected_bytes()
+    ctx_tokens = int(ds.ctx_lens.sum().item())
+    dense_bytes = ctx_tokens * ds.wl.kv_bytes_per_token()
+
+    res = {"selected_bytes": sel, "dense_bytes": dense_bytes, "density": sel / max(dense_bytes, 1),
+           "kv_copies": ncopy, "launches_per_step": launches_per_step, "dev_status": status}
+
+    # (a) direct calls through the binding
+    ms = timer.run(lambda i: (rot(i), ds.step()), steps)
+    res["direct_us"] = ms / steps * 1e3
+    # (b) the same step replayed from CUDA graphs (one per KV copy)
+    graphs = capture_graphs(torch, ds, ds.step)
+    for g in graphs:
+        g.replay()
+    ms = timer.run(lambda i: graphs[i % ncopy].replay(), steps)
+    res["graph_us"] = ms / steps * 1e3
+    # (c) pieces, from graphs as well: index alone, attention alone, dense alone
+    for name, fn in (("index_us", ds.build_index), ("sparse_attn_us", ds.attend_sparse),
+                     ("dense_us", ds.attend_dense)):
+        gs = capture_graphs(torch, ds, fn)
+        for g in gs:
+            g.replay()
+        n = steps if name != "dense_us" else max(10, min(steps, int(steps * sel / max(dense_bytes, 1)) + 10))
+        ms = timer.run(lambda i: gs[i % ncopy].replay(), n)
+        res[name] = ms / n * 1e3
+        del gs
+    ds.step()                                   # leave the sparse result in place
+    # (d) the main kernel alone: events recorded by the library around it
+    if kernel_pass:
+        n = min(steps, 500)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b in evs:
+            a.record()
+            b.record()
+        torch.cuda.synchronize()
+
+        def with_events(i):
+            rot(i)
+            ds.build_index()
+            ssa.set_kernel_events(*evs[i])
+            ds.attend_sparse()
+
+        timer.run(with_events, n)
+        durs = [a.elapsed_time(b) for a, b in evs]
+        res["kernel_us"] = statistics.mean(durs) * 1e3
+        res["kernel_us_median"] = statistics.median(durs) * 1e3
+    step_us = min(res["graph_us"], res["direct_us"])
+    res["step_us"] = step_us
+    res["launch_mode"] = "cuda_graph" if res["graph_us"] <= res["direct_us"] else "direct"
+    res["gbs"] = sel / step_us / 1e3
+    res["pct_peak_measured"] = 100 * res["gbs"] / peak
+    res["pct_peak_spec"] = 100 * res["gbs"] / SPEC_HBM_GBS
+    res["attn_gbs"] = sel / res["sparse_attn_us"] / 1e3
+    res["dense_gbs"] = dense_bytes / res["dense_us"] / 1e3
+    res["speedup_vs_dense"] = res["dense_us"] / step_us
+    return res
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2404_09336_b200 import inputs, ssa
+    from paper_2404_09336_b200.runner import DecodeStep
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peak, peak_kind = hbm_peak()
+    timer = Timer(torch, dist, world)
+    l2 = l2_bytes(torch)
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    try:
+        gpu_id = f"GPU-{torch.cuda.get_device_properties(local).uuid}"
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    density = 0.10 if args.cfg == 5 else None
+    wl = inputs.make_config(args.cfg, density=density, first_id=rank * 1000)
+    sel_guess = wl.selected_upper_bound() * wl.B * wl.kv_bytes_per_token() // 2
+    cache = 2 * wl.B * wl.H * wl.max_ctx * wl.D * 2
+    ds = DecodeStep(wl, device=f"cuda:{local}", kv_copies=copies_for(sel_guess, cache, l2))
+    main = measure(torch, ssa, timer, ds, steps, warmup, peak)
+    if main["dev_status"] != 0:
+        raise SystemExit(f"device status word is {main['dev_status']}: the workload raised a data flag")
+
+    # the headline region once more, as the explicit K-step timed loop
+    ncopy = len(ds.k_store)
+    graphs = capture_graphs(torch, ds, ds.step)
+    for g in graphs:
+        g.replay()
+    use_graph = main["launch_mode"] == "cuda_graph"
+    l0 = ssa.launch_count()
+    if use_graph:
+        ms = timer.run(lambda i: graphs[i % ncopy].replay(), steps)
+        launches = steps * main["launches_per_step"]
+    else:
+        ms = timer.run(lambda i: (ds.select_copy(i % ncopy), ds.step()), steps)
+        launches = ssa.launch_count() - l0
+    total_sel = timer.total(main["selected_bytes"])
+    value = total_sel * steps / (ms * 1e-3) / 1e9
+
+    # end to end: per-step inputs from pinned host memory, result back to the host
+    h2d, d2h = ds.make_host_buffers()
+    for i in range(3):
+        ds.step_from_host()
+    ms_e2e = timer.run(lambda i: (ds.select_copy(i % ncopy), ds.step_from_host()), steps)
+    e2e_value = total_sel * steps / (ms_e2e * 1e-3) / 1e9
+    clocks = sampler.stop(timer.windows)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    kernel_us = main.get("kernel_us")
+    roofline = {"bound": "hbm", "kernel": "decode_partial_kernel (sparse)",
+                "achieved": main["selected_bytes"] / kernel_us / 1e3 if kernel_us else None,
+                "peak": peak, "unit": "GB/s", "peak_kind": f"of {peak_kind}",
+                "frac": (main["selected_bytes"] / kernel_us / 1e3 / peak) if kernel_us else None,
+                "frac_of_spec_8000": (main["selected_bytes"] / kernel_us / 1e3 / SPEC_HBM_GBS) if kernel_us else None,
+                "traffic": None, "kernel_us": kernel_us,
+                "algorithmic_bytes_per_launch": main["selected_bytes"]}
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.cfg] + (" (10% point)" if args.cfg == 5 else ""),
+                   "layout": "[B,H,T,D]", "kv_dtype": wl.dtype, "launch": main["launch_mode"],
+                   "l2": f"inputs larger than L2: {ncopy} rotating KV copies, "
+                         f"{ncopy * main['selected_bytes'] / 1e6:.0f} MB of selected rows between reuses "
+                         f"(L2 {l2 / 1e6:.0f} MB)",
+                   "per_gpu_batch": wl.B},
+        "pct_hbm_peak_measured": 100 * value / world / peak, "pct_hbm_peak_spec": 100 * value / world / SPEC_HBM_GBS,
+        "speedup_vs_dense": main["speedup_vs_dense"], "density": main["density"],
+        "us_per_step": ms / steps * 1e3,
+        "breakdown_us": {k: main[k] for k in ("direct_us", "graph_us", "index_us", "sparse_attn_us", "dense_us")},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "us_per_step": ms_e2e / steps * 1e3,
+                "note": "query rows + span lists copied in from pinned memory, output rows + counts + status "
+                        "copied back; the KV cache is resident state"},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+    }
+
+    if world == 1:
+        del graphs
+        sweep = []
+        want = {"auto": [3, 4, 5], "all": [1, 3, 4, 5], "none": []}[args.sweep]
+        sweep_steps = max(20, min(steps, 200))
+        del ds
+        torch.cuda.empty_cache()
+        for cfg in want:
+            if cfg == args.cfg:
+                continue
+            if cfg == 5:
+                wls = {f: inputs.make_config(5, density=f) for f in inputs.DENSITIES}
+                cap = max(len(w.spans) for w in wls.values())
+                d5 = DecodeStep(wls[1.0], kv_copies=6, index_stride=8192, max_selected=8192, span_capacity=cap)
+                for f in inputs.DENSITIES:
+                    d5.set_spans(wls[f])
+                    r = measure(torch, ssa, timer, d5, sweep_steps, 3, peak, kernel_pass=False)
+                    r["workload"] = f"cfg5 density {int(f * 100)}%"
+                    sweep.append(r)
+                del d5
+            else:
+                w = inputs.make_config(cfg)
+                sg = w.selected_upper_bound() * w.B * w.kv_bytes_per_token() // 2
+                cb = 2 * w.B * w.H * w.max_ctx * w.D * 2
+                d = DecodeStep(w, kv_copies=copies_for(sg, cb, l2))
+                r = measure(torch, ssa, timer, d, sweep_steps, 3, peak, kernel_pass=False)
+                r["workload"] = WORKLOAD_TEXT[cfg].split(":")[0]
+                sweep.append(r)
+                del d
+            torch.cuda.empty_cache()
+        keep = ("workload", "density", "selected_bytes", "step_us", "index_us", "sparse_attn_us", "dense_us", "gbs",
+                "attn_gbs", "dense_gbs", "pct_peak_measured", "pct_peak_spec", "speedup_vs_dense", "launch_mode",
+                "kv_copies")
+        line["sweep"] = [{k: (round(r[k], 4) if isinstance(r[k], float) else r[k]) for k in keep} for r in sweep]
+        five = [r for r in sweep if r["workload"].startswith("cfg5")]
+        cross = next((r["density"] for r in five if r["speedup_vs_dense"] < 1.0), None)
+        line["crossover_density"] = cross
+        line["cpu_baseline"] = time_oracle(args.cfg, budget_s=15.0)
+        for k in ("seconds", "ms_per_step", "steps"):
+            line["cpu_baseline"].pop(k, None)
+    else:
+        dist.barrier()
+        dist.destroy_process_group()
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cfg", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--sweep", default="auto", choices=["auto", "none", "all"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

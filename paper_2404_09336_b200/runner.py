@@ -26,6 +26,22 @@ def tensor_to_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
+def _arena(device, specs):
+    """One uint8 device buffer holding tensors of the given (shape, dtype)
+    back to back at 256-byte boundaries; returns (buffer, views)."""
+    offs, total = [], 0
+    for shape, dt in specs:
+        offs.append(total)
+        nbytes = int(np.prod(shape)) * torch.empty((), dtype=dt).element_size()
+        total += (nbytes + 255) // 256 * 256
+    buf = torch.zeros(total, dtype=torch.uint8, device=device)
+    views = []
+    for (shape, dt), o in zip(specs, offs):
+        nbytes = int(np.prod(shape)) * torch.empty((), dtype=dt).element_size()
+        views.append(buf[o:o + nbytes].view(dt).view(shape))
+    return buf, views
+
+
 class DecodeStep:
     """Buffers of one workload on one GPU.
 
@@ -37,12 +53,12 @@ class DecodeStep:
     """
 
     def __init__(self, wl: Workload, device="cuda:0", layout="bhtd", out_dtype=None, kv_copies=1,
-                 index_stride=None, max_selected=None, gen_threads=None):
+                 index_stride=None, max_selected=None, gen_threads=None,
+                 span_capacity=0):
         self.wl, self.device, self.layout = wl, torch.device(device), layout
         dt = _TORCH_DTYPE[wl.dtype]
         dev = self.device
         B, H, D, T = wl.B, wl.H, wl.D, wl.max_ctx
-        self.q = bits_to_tensor(wl.q_bits(), wl.dtype).to(dev)
         shape = (B, H, T, D) if layout == "bhtd" else (B, T, H, D)
         self.k_store = [torch.empty(shape, dtype=dt, device=dev) for _ in range(kv_copies)]
         self.v_store = [torch.empty(shape, dtype=dt, device=dev) for _ in range(kv_copies)]
@@ -65,17 +81,25 @@ class DecodeStep:
             self.k_store[c].copy_(self.k_store[0])
             self.v_store[c].copy_(self.v_store[0])
         self.select_copy(0)
-        self.ctx_lens = torch.from_numpy(wl.ctx_lens.copy()).to(dev)
-        self.span_offsets = torch.from_numpy(wl.span_offsets.copy()).to(dev)
         spans = wl.spans if len(wl.spans) else np.zeros((1, 2), np.int32)
-        self.spans = torch.from_numpy(np.ascontiguousarray(spans)).to(dev)
         self.max_selected = int(max_selected or max(wl.selected_upper_bound(), 1))
         self.index_stride = int(index_stride or (self.max_selected + 31) // 32 * 32)
+        odt = out_dtype or dt
+        # what changes every decode step lives in one input arena and one result
+        # arena, so that a host-driven step is one copy in and one copy out
+        self.in_arena, (self.q, self.ctx_lens, self.span_offsets, self.spans) = _arena(
+            dev, [((B, H, D), dt), ((B,), torch.int32), ((B + 1,), torch.int32), ((max(len(spans), span_capacity), 2), torch.int32)])
+        self.out_arena, (self.out, self.lse, self.counts, self.status) = _arena(
+            dev, [((B, H, D), odt), ((B, H), torch.float32), ((B,), torch.int32), ((1,), torch.int32)])
+        self.q.copy_(bits_to_tensor(wl.q_bits(), wl.dtype))
+        self.ctx_lens.copy_(torch.from_numpy(wl.ctx_lens.copy()))
+        self.span_offsets.copy_(torch.from_numpy(wl.span_offsets.copy()))
+        self.spans[: len(spans)].copy_(torch.from_numpy(np.ascontiguousarray(spans)))
+        self.out.zero_()
+        self.lse.zero_()
+        self.counts.fill_(-7)
+        self.status.zero_()
         self.index = torch.full((B, self.index_stride), -7, dtype=torch.int32, device=dev)
-        self.counts = torch.full((B,), -7, dtype=torch.int32, device=dev)
-        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.out = torch.zeros((B, H, D), dtype=out_dtype or dt, device=dev)
-        self.lse = torch.zeros((B, H), dtype=torch.float32, device=dev)
         self.desc = ssa.make_desc(self.q, self.k, self.v, self.out, max_ctx=T)
         need = max(ssa.decode_workspace_bytes(self.desc, self.max_selected),
                    ssa.decode_workspace_bytes(self.desc, T))
@@ -109,30 +133,30 @@ class DecodeStep:
 
     # ---- host-buffer form (end-to-end timing) -----------------------------------------
     def make_host_buffers(self):
-        """Pinned host copies of what changes every decode step (query rows and
-        span lists) and pinned landing buffers for what the caller reads back.
+        """Pinned host copy of what changes every decode step (query rows,
+        context lengths, span lists) and a pinned landing buffer for what the
+        caller reads back (output rows, lse, counts, status word).
         Returns (host-to-device bytes, device-to-host bytes) per step."""
-        pin = lambda t: t.detach().cpu().pin_memory()
-        self.h_q, self.h_spans = pin(self.q), pin(self.spans)
-        self.h_offsets, self.h_ctx = pin(self.span_offsets), pin(self.ctx_lens)
-        self.h_out = torch.empty(self.out.shape, dtype=self.out.dtype).pin_memory()
-        self.h_counts = torch.empty(self.counts.shape, dtype=torch.int32).pin_memory()
-        self.h_status = torch.empty(1, dtype=torch.int32).pin_memory()
-        h2d = sum(t.numel() * t.element_size() for t in (self.h_q, self.h_spans, self.h_offsets, self.h_ctx))
-        d2h = sum(t.numel() * t.element_size() for t in (self.h_out, self.h_counts, self.h_status))
-        return h2d, d2h
+        self.h_in = self.in_arena.cpu().pin_memory()
+        self.h_out = torch.empty(self.out_arena.shape, dtype=torch.uint8).pin_memory()
+        return self.h_in.numel(), self.h_out.numel()
 
     def step_from_host(self, stream=None):
-        """Decode step whose per-step inputs start in (pinned) host memory and
+        """Decode step whose per-step inputs start in pinned host memory and
         whose result ends there; the KV cache is the resident state."""
-        self.q.copy_(self.h_q, non_blocking=True)
-        self.spans.copy_(self.h_spans, non_blocking=True)
-        self.span_offsets.copy_(self.h_offsets, non_blocking=True)
-        self.ctx_lens.copy_(self.h_ctx, non_blocking=True)
+        self.in_arena.copy_(self.h_in, non_blocking=True)
         self.step(stream)
-        self.h_out.copy_(self.out, non_blocking=True)
-        self.h_counts.copy_(self.counts, non_blocking=True)
-        self.h_status.copy_(self.status, non_blocking=True)
+        self.h_out.copy_(self.out_arena, non_blocking=True)
+
+    def set_spans(self, wl: Workload):
+        """Replace the span lists (same geometry, same cache)."""
+        assert (wl.B, wl.H, wl.D, wl.max_ctx) == (self.wl.B, self.wl.H, self.wl.D, self.wl.max_ctx)
+        assert wl.spans.shape[0] <= self.spans.shape[0] and wl.selected_upper_bound() <= self.index_stride
+        self.spans[: wl.spans.shape[0]].copy_(torch.from_numpy(np.ascontiguousarray(wl.spans)))
+        self.span_offsets.copy_(torch.from_numpy(wl.span_offsets.copy()))
+        self.ctx_lens.copy_(torch.from_numpy(wl.ctx_lens.copy()))
+        self.max_selected = max(wl.selected_upper_bound(), 1)
+        self.wl = wl
 
     # ---- results ---------------------------------------------------------------------
     def out_f64(self) -> np.ndarray:

@@ -92,6 +92,12 @@ def _stream(stream):
     return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
 
 
+def _row_stride(index):
+    """Elements between consecutive rows of index[B, n] (a one-row tensor may
+    carry an arbitrary stride for its size-1 dimension)."""
+    return int(index.stride(0) if index.shape[0] > 1 else index.shape[1])
+
+
 def _check(fn, rc, check):
     if check and rc != OK:
         raise SsaError(fn, rc)
@@ -121,7 +127,7 @@ def make_desc(q, k_cache, v_cache, out, max_ctx=None, scale: float = 0.0) -> Att
 def spans_to_index(span_offsets, spans, ctx_lens, index, counts, dev_status=None, stream=None, check=True):
     """ssa_spans_to_index: index[B, index_stride] and counts[B] are written."""
     rc = lib.ssa_spans_to_index(_ptr(span_offsets), _ptr(spans), _ptr(ctx_lens), int(ctx_lens.numel()),
-                                _ptr(index), int(index.stride(0)), _ptr(counts), _ptr(dev_status),
+                                _ptr(index), _row_stride(index), _ptr(counts), _ptr(dev_status),
                                 _stream(stream))
     return _check("ssa_spans_to_index", rc, check)
 
@@ -135,7 +141,7 @@ def decode_attn_sparse(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_s
     """ssa_decode_attn_sparse: out (and lse) are written."""
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     rc = lib.ssa_decode_attn_sparse(C.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens),
-                                    _ptr(index), int(index.stride(0)) if index is not None else 0,
+                                    _ptr(index), _row_stride(index) if index is not None else 0,
                                     _ptr(counts), int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace),
                                     ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_sparse", rc, check)
