@@ -4,15 +4,17 @@
 // Pass 1 (decode_partial_kernel): grid (chunk, head, request).  A block owns
 // `chunk` consecutive entries of the request's index list (dense: `chunk`
 // consecutive positions).  A cache row of D 16-bit values is read by a group
-// of D/8 lanes with one 16-byte load per lane, so a warp covers 32/(D/8) rows
-// per load instruction and every 32-byte sector of a selected row is fetched
-// exactly once.  Each lane keeps kU K-loads and kU V-loads in flight, then
-// reduces the kU dot products across its lane group with shuffles and folds
+// of D/16 lanes, 32 bytes per lane (one 256-bit load where the cache is
+// 32-byte aligned, else two 128-bit loads), so a warp covers 32/(D/16) rows
+// per load and every 32-byte sector of a selected row is fetched exactly once.
+// A warp keeps a tile of kU such loads of K and kU of V in flight, then
+// reduces the kU dot products across each lane group with shuffles and folds
 // them into a running (max, sum, accumulator) triple - the online form of the
-// softmax.  Lane groups never talk to one another until the block ends, where
-// their triples are combined through shared memory.  With one chunk per
-// request the block normalises and stores the output itself; otherwise it
-// stores the unnormalised triple to the workspace and
+// softmax.  The arithmetic is packed: two fp32 lanes per FMA (fma.rn.f32x2).
+// Lane groups never talk to one another until the block ends, where their
+// triples are combined through shared memory.  With one chunk per request the
+// block normalises and stores the output itself; otherwise it stores the
+// unnormalised triple to the workspace and
 // Pass 2 (decode_merge_kernel) combines the chunks of one (request, head).
 #include "ssa_common.cuh"
 
@@ -22,13 +24,17 @@ namespace ssa {
 #define SSA_WARPS 4
 #endif
 #ifndef SSA_U
-#define SSA_U 8
+#define SSA_U 4
+#endif
+#ifndef SSA_MIN_BLOCKS
+#define SSA_MIN_BLOCKS 4
 #endif
 
 constexpr int kWarps = SSA_WARPS;      // warps per block in pass 1
 constexpr int kThreads = kWarps * 32;
-constexpr int kU = SSA_U;              // row loads in flight per lane, per tensor
-constexpr int kMaxChunk = 1024;        // index entries staged per block
+constexpr int kU = SSA_U;              // 32-byte loads in flight per lane, per tensor
+constexpr int kMaxChunk = 512;         // index entries staged per block
+constexpr int kIdxPerThread = kMaxChunk / kThreads;
 
 struct DecodeParams {
   const void* q;
@@ -42,7 +48,8 @@ struct DecodeParams {
   float* ws_acc;            // [B*H*n_chunks, D]
   float2* ws_ml;            // [B*H*n_chunks]  (max in log2 units, sum)
   uint32_t* dev_status;
-  int64_t q_sb, q_sh, k_sb, k_st, k_sh, v_sb, v_st, v_sh, o_sb, o_sh;
+  int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;
+  uint32_t k_row_bytes, v_row_bytes;   // token stride of the cache in bytes
   int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32;
   float scale_log2;         // softmax scale * log2(e)
 };
@@ -70,10 +77,32 @@ __device__ __forceinline__ void store_out(const DecodeParams& p, int b, int h, i
   else reinterpret_cast<T*>(p.out)[o] = from_float<T>(val);
 }
 
-template <typename T, int D, bool kSparse>
-__global__ void __launch_bounds__(kThreads)
+// 32 bytes of a cache row: eight packed pairs of 16-bit values.
+struct Piece { uint32_t w[8]; };
+
+template <bool kAligned32>
+__device__ __forceinline__ void load_piece(Piece& r, const char* p) {
+  if (kAligned32) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]),
+                   "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+                 : "l"(p));
+  } else {
+    const uint4 a = ld_stream_16B(p), b = ld_stream_16B(p + 16);
+    r.w[0] = a.x; r.w[1] = a.y; r.w[2] = a.z; r.w[3] = a.w;
+    r.w[4] = b.x; r.w[5] = b.y; r.w[6] = b.z; r.w[7] = b.w;
+  }
+}
+
+__device__ __forceinline__ void zero_piece(Piece& r) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) r.w[i] = 0u;
+}
+
+template <typename T, int D, bool kSparse, bool kAligned32>
+__global__ void __launch_bounds__(kThreads, SSA_MIN_BLOCKS)
 decode_partial_kernel(const DecodeParams p) {
-  constexpr int kLanesPerRow = D / 8;                 // 16-byte pieces per row
+  constexpr int kLanesPerRow = D / 16;                // 32-byte pieces per row
   constexpr int kRowsPerLoad = 32 / kLanesPerRow;     // rows one warp-wide load covers
   constexpr int kTileRows = kRowsPerLoad * kU;        // rows per warp per iteration
   constexpr int kGroups = kWarps * kRowsPerLoad;      // independent softmax streams
@@ -82,102 +111,139 @@ decode_partial_kernel(const DecodeParams p) {
   __shared__ int32_t s_idx[kSparse ? kMaxChunk : 1];
   __shared__ __align__(16) float s_acc[kGroups][D];
   __shared__ float s_m[kGroups], s_l[kGroups];
+  __shared__ int s_bad;
 
   const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int col = lane % kLanesPerRow, sub = lane / kLanesPerRow;
+  const int start = chunk_id * p.chunk;
+
+  // Everything the block needs before it can request cache rows is loaded
+  // here in one go: sizes, its slice of the index list, the query row.
+  int32_t raw[kIdxPerThread];
+  if (kSparse) {
+    const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
+#pragma unroll
+    for (int j = 0; j < kIdxPerThread; ++j) {
+      const int i = tid + j * kThreads;
+      raw[j] = (i < p.chunk && start + i < p.max_selected) ? __ldg(row + i) : -1;
+    }
+    if (tid == 0) s_bad = 0;
+  }
+  Piece qraw;
+  load_piece<false>(qraw, reinterpret_cast<const char*>(
+      reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + col * 16));
 
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
-  const int start = chunk_id * p.chunk;
   if (start >= c && chunk_id > 0) return;             // chunk 0 always reports
   const int cnt = max(0, min(p.chunk, c - start));
 
   if (kSparse) {
-    const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
-    for (int i = tid; i < cnt; i += kThreads) {
-      int v = row[i];
-      if (v < 0 || v >= n) { v = -1; flags |= SSA_DEV_BAD_INDEX; }
-      s_idx[i] = v;
+    __syncthreads();                                  // s_bad cleared
+#pragma unroll
+    for (int j = 0; j < kIdxPerThread; ++j) {
+      const int i = tid + j * kThreads;
+      if (i < cnt) {
+        int v = raw[j];
+        if (v < 0 || v >= n) { v = -1; flags |= SSA_DEV_BAD_INDEX; s_bad = 1; }
+        s_idx[i] = v;
+      }
     }
+    __syncthreads();
   }
   if (p.dev_status && h == 0) {
     const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
     if (f) atomicOr(p.dev_status, f);
   }
+  const bool any_bad = kSparse ? (s_bad != 0) : false;
 
-  float qf[8];
-  {
-    const T* qp = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + col * 8;
-    unpack8<T>(*reinterpret_cast<const uint4*>(qp), qf);
+  const char* kbase = reinterpret_cast<const char*>(
+      reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)h * p.k_sh + col * 16);
+  const char* vbase = reinterpret_cast<const char*>(
+      reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)h * p.v_sh + col * 16);
+
+  float2 q2[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) qf[i] *= p.scale_log2;
+  for (int i = 0; i < 8; ++i) {
+    q2[i] = unpack2<T>(qraw.w[i]);
+    q2[i].x *= p.scale_log2;
+    q2[i].y *= p.scale_log2;
   }
-  if (kSparse) __syncthreads();
-
-  const T* kbase = reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)h * p.k_sh + col * 8;
-  const T* vbase = reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)h * p.v_sh + col * 8;
-
   float m = neg_inf(), l = 0.f;
-  float acc[8];
+  float2 acc[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+  for (int i = 0; i < 8; ++i) acc[i] = make_float2(0.f, 0.f);
 
   for (int t = warp * kTileRows; t < cnt; t += kWarps * kTileRows) {
-    uint4 kr[kU], vr[kU];
-    bool ok[kU];
+    Piece kr[kU], vr[kU];
+    float s[kU];
+    // full tiles without bad entries take the unpredicated path
+    const bool checked = any_bad || (t + kTileRows > cnt);
+    if (!checked) {
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const int r = t + u * kRowsPerLoad + sub;
-      int pos = -1;
-      if (r < cnt) pos = kSparse ? s_idx[r] : start + r;
-      ok[u] = pos >= 0;
-      if (ok[u]) {
-        kr[u] = ld_stream_16B(kbase + (int64_t)pos * p.k_st);
-        vr[u] = ld_stream_16B(vbase + (int64_t)pos * p.v_st);
-      } else {
-        kr[u] = make_uint4(0, 0, 0, 0);
-        vr[u] = make_uint4(0, 0, 0, 0);
+      for (int u = 0; u < kU; ++u) {
+        const int r = t + u * kRowsPerLoad + sub;
+        const uint32_t pos = (uint32_t)(kSparse ? s_idx[r] : start + r);
+        load_piece<kAligned32>(kr[u], kbase + (uint64_t)pos * p.k_row_bytes);
+        load_piece<kAligned32>(vr[u], vbase + (uint64_t)pos * p.v_row_bytes);
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+        const int r = t + u * kRowsPerLoad + sub;
+        int pos = -1;
+        if (r < cnt) pos = kSparse ? s_idx[r] : start + r;
+        if (pos >= 0) {
+          load_piece<kAligned32>(kr[u], kbase + (uint64_t)(uint32_t)pos * p.k_row_bytes);
+          load_piece<kAligned32>(vr[u], vbase + (uint64_t)(uint32_t)pos * p.v_row_bytes);
+          s[u] = 0.f;
+        } else {
+          zero_piece(kr[u]);
+          zero_piece(vr[u]);
+          s[u] = neg_inf();                           // marks the row as masked
+        }
       }
     }
-    float s[kU];
     float mt = neg_inf();
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-      float kf[8];
-      unpack8<T>(kr[u], kf);
-      float d = 0.f;
+      float2 d2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) d = fmaf(qf[i], kf[i], d);
+      for (int i = 0; i < 8; ++i) d2 = fma2(q2[i], unpack2<T>(kr[u].w[i]), d2);
+      float d = d2.x + d2.y;
 #pragma unroll
       for (int o = kLanesPerRow / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-      s[u] = ok[u] ? d : neg_inf();
+      s[u] = checked ? d + s[u] : d;                  // -inf stays -inf
       mt = fmaxf(mt, s[u]);
     }
     const float m_new = fmaxf(m, mt);
     if (m_new > neg_inf()) {
-      const float alpha = fast_exp2(m - m_new);       // m = -inf gives 0
-      l *= alpha;
+      if (m_new > m) {                                // rare after the first tiles
+        const float alpha = fast_exp2(m - m_new);     // m = -inf gives 0
+        l *= alpha;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] *= alpha;
+        for (int i = 0; i < 8; ++i) { acc[i].x *= alpha; acc[i].y *= alpha; }
+        m = m_new;
+      }
 #pragma unroll
       for (int u = 0; u < kU; ++u) {
-        const float pw = fast_exp2(s[u] - m_new);     // masked rows give 0
+        const float pw = fast_exp2(s[u] - m);         // masked rows give 0
         l += pw;
-        float vf[8];
-        unpack8<T>(vr[u], vf);
+        const float2 pw2 = make_float2(pw, pw);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = fmaf(pw, vf[i], acc[i]);
+        for (int i = 0; i < 8; ++i) acc[i] = fma2(pw2, unpack2<T>(vr[u].w[i]), acc[i]);
       }
-      m = m_new;
     }
   }
 
   // combine the lane groups of the block
   const int g = warp * kRowsPerLoad + sub;
-  *reinterpret_cast<float4*>(&s_acc[g][col * 8]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-  *reinterpret_cast<float4*>(&s_acc[g][col * 8 + 4]) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    *reinterpret_cast<float4*>(&s_acc[g][col * 16 + 4 * i]) =
+        make_float4(acc[2 * i].x, acc[2 * i].y, acc[2 * i + 1].x, acc[2 * i + 1].y);
   if (col == 0) { s_m[g] = m; s_l[g] = l; }
   __syncthreads();
   if (tid < D) {
@@ -259,17 +325,23 @@ static int32_t check_desc(const ssa_attn_desc* d) {
     if (s < 0) return SSA_ERR_SHAPE;
     if (s % 8 != 0) return SSA_ERR_ALIGN;
   }
+  if (d->k_stride_t >= (1ll << 31) || d->v_stride_t >= (1ll << 31)) return SSA_ERR_SHAPE;
   return SSA_OK;
 }
 
 template <typename T, int D>
-static int32_t launch(const DecodeParams& p, int B, bool sparse, cudaStream_t st) {
+static int32_t launch(const DecodeParams& p, int B, bool sparse, bool aligned32, cudaStream_t st) {
   cudaEvent_t ev_b, ev_e;
   take_kernel_events(&ev_b, &ev_e);
   dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
   if (ev_b) cudaEventRecord(ev_b, st);
-  if (sparse) decode_partial_kernel<T, D, true><<<grid, kThreads, 0, st>>>(p);
-  else decode_partial_kernel<T, D, false><<<grid, kThreads, 0, st>>>(p);
+  if (sparse) {
+    if (aligned32) decode_partial_kernel<T, D, true, true><<<grid, kThreads, 0, st>>>(p);
+    else decode_partial_kernel<T, D, true, false><<<grid, kThreads, 0, st>>>(p);
+  } else {
+    if (aligned32) decode_partial_kernel<T, D, false, true><<<grid, kThreads, 0, st>>>(p);
+    else decode_partial_kernel<T, D, false, false><<<grid, kThreads, 0, st>>>(p);
+  }
   if (ev_e) cudaEventRecord(ev_e, st);
   if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   int launches = 1;
@@ -310,8 +382,10 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   p.ws_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(ws) + pl.acc_bytes);
   p.dev_status = dev_status;
   p.q_sb = d->q_stride_b; p.q_sh = d->q_stride_h;
-  p.k_sb = d->k_stride_b; p.k_st = d->k_stride_t; p.k_sh = d->k_stride_h;
-  p.v_sb = d->v_stride_b; p.v_st = d->v_stride_t; p.v_sh = d->v_stride_h;
+  p.k_sb = d->k_stride_b; p.k_sh = d->k_stride_h;
+  p.v_sb = d->v_stride_b; p.v_sh = d->v_stride_h;
+  p.k_row_bytes = (uint32_t)(d->k_stride_t * 2);
+  p.v_row_bytes = (uint32_t)(d->v_stride_t * 2);
   p.o_sb = d->o_stride_b; p.o_sh = d->o_stride_h;
   p.H = d->H; p.max_ctx = d->max_ctx;
   p.index_stride = index_stride; p.max_selected = max_selected;
@@ -320,10 +394,15 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->D);
   p.scale_log2 = scale * kLog2e;
 
+  // one 256-bit load per lane needs every cache row piece on a 32-byte boundary
+  const bool a32 = reinterpret_cast<uintptr_t>(k) % 32 == 0 && reinterpret_cast<uintptr_t>(v) % 32 == 0 &&
+                   d->k_stride_b % 16 == 0 && d->k_stride_t % 16 == 0 && d->k_stride_h % 16 == 0 &&
+                   d->v_stride_b % 16 == 0 && d->v_stride_t % 16 == 0 && d->v_stride_h % 16 == 0;
   cudaStream_t st = (cudaStream_t)stream;
   if (d->kv_dtype == SSA_BF16)
-    return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, sparse, st) : launch<__nv_bfloat16, 64>(p, d->B, sparse, st);
-  return d->D == 128 ? launch<__half, 128>(p, d->B, sparse, st) : launch<__half, 64>(p, d->B, sparse, st);
+    return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, sparse, a32, st)
+                       : launch<__nv_bfloat16, 64>(p, d->B, sparse, a32, st);
+  return d->D == 128 ? launch<__half, 128>(p, d->B, sparse, a32, st) : launch<__half, 64>(p, d->B, sparse, a32, st);
 }
 
 }  // namespace ssa
