@@ -3,7 +3,8 @@
 // One thread block per (output slice, request).  The block
 //   1. loads the request's spans, clamps them to [0, ctx_len) and packs each
 //      non-empty one into a 64-bit key (start << 32 | end);
-//   2. sorts the keys (bitonic network in shared memory);
+//   2. sorts the keys: up to 32 spans by rank counting inside one warp
+//      (shuffles only), more by a bitonic network in shared memory;
 //   3. has one warp walk the sorted spans 32 at a time with two shuffle
 //      scans: a running maximum of the span ends seen so far, which trims
 //      each span to the part no earlier span covers, and a prefix sum of the
@@ -17,7 +18,7 @@
 
 namespace ssa {
 
-constexpr int kIdxThreads = 256;
+constexpr int kIdxThreads = 128;
 constexpr int kMaxSpans = SSA_MAX_SPANS_PER_SEQ;   // power of two
 constexpr unsigned long long kEmptyKey = 0xffffffffffffffffull;
 
@@ -42,33 +43,49 @@ spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* _
   int P = 32;
   while (P < S) P <<= 1;
   if (tid == 0) s_flags = 0;
-
-  // 1. load, clamp, pack
-  for (int i = tid; i < P; i += kIdxThreads) {
-    unsigned long long key = kEmptyKey;
-    if (i < S) {
-      const int2 se = reinterpret_cast<const int2*>(spans)[first + i];
-      if (se.x < 0 || se.x > se.y) flags |= SSA_DEV_BAD_SPAN;
-      if (se.y > n) flags |= SSA_DEV_CLIPPED;
-      const int s = max(se.x, 0), e = min(se.y, n);
-      if (e > s) key = ((unsigned long long)(uint32_t)s << 32) | (uint32_t)e;
-    }
-    keys[i] = key;
-  }
   __syncthreads();
 
-  // 2. bitonic sort, ascending by (start, end); empty keys sink to the end
-  for (int k = 2; k <= P; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < P; i += kIdxThreads) {
-        const int ixj = i ^ j;
-        if (ixj > i) {
-          const unsigned long long a = keys[i], c = keys[ixj];
-          const bool up = (i & k) == 0;
-          if ((a > c) == up) { keys[i] = c; keys[ixj] = a; }
-        }
+  // clamp a span to the context and pack it; empty spans get the sentinel
+  auto load_key = [&](int i) -> unsigned long long {
+    if (i >= S) return kEmptyKey;
+    const int2 se = reinterpret_cast<const int2*>(spans)[first + i];
+    if (se.x < 0 || se.x > se.y) flags |= SSA_DEV_BAD_SPAN;
+    if (se.y > n) flags |= SSA_DEV_CLIPPED;
+    const int s = max(se.x, 0), e = min(se.y, n);
+    return e > s ? ((unsigned long long)(uint32_t)s << 32) | (uint32_t)e : kEmptyKey;
+  };
+
+  if (P == 32) {
+    // 1+2 (up to 32 spans, the usual case): one warp ranks its keys with
+    // shuffles, no block barrier needed
+    if (tid < 32) {
+      const unsigned long long key = load_key(tid);
+      int rank = 0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const unsigned long long kj = __shfl_sync(0xffffffffu, key, j);
+        rank += (kj < key || (kj == key && j < tid)) ? 1 : 0;
       }
-      __syncthreads();
+      keys[rank] = key;
+      __syncwarp();
+    }
+  } else {
+    // 1. load, clamp, pack
+    for (int i = tid; i < P; i += kIdxThreads) keys[i] = load_key(i);
+    __syncthreads();
+    // 2. bitonic sort, ascending by (start, end); empty keys sink to the end
+    for (int k = 2; k <= P; k <<= 1) {
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int i = tid; i < P; i += kIdxThreads) {
+          const int ixj = i ^ j;
+          if (ixj > i) {
+            const unsigned long long a = keys[i], c = keys[ixj];
+            const bool up = (i & k) == 0;
+            if ((a > c) == up) { keys[i] = c; keys[ixj] = a; }
+          }
+        }
+        __syncthreads();
+      }
     }
   }
 
