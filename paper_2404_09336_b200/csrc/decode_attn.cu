@@ -118,6 +118,8 @@ decode_partial_kernel(const DecodeParams p) {
   const int col = lane % kLanesPerRow, sub = lane / kLanesPerRow;
   const int start = chunk_id * p.chunk;
 
+  grid_dependency_wait();
+
   // Everything the block needs before it can request cache rows is loaded
   // here in one go: sizes, its slice of the index list, the query row.
   int32_t raw[kIdxPerThread];
@@ -238,6 +240,10 @@ decode_partial_kernel(const DecodeParams p) {
     }
   }
 
+  // all cache rows of this block have been read: the next kernel of the stream
+  // may start filling the SMs this grid is leaving
+  grid_launch_dependents();
+
   // combine the lane groups of the block
   const int g = warp * kRowsPerLoad + sub;
 #pragma unroll
@@ -272,6 +278,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(D)
 decode_merge_kernel(const DecodeParams p) {
   const int h = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
+  grid_dependency_wait();
+  grid_launch_dependents();
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
@@ -334,20 +342,17 @@ static int32_t launch(const DecodeParams& p, int B, bool sparse, bool aligned32,
   cudaEvent_t ev_b, ev_e;
   take_kernel_events(&ev_b, &ev_e);
   dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
+  void (*kernel)(const DecodeParams) =
+      sparse ? (aligned32 ? decode_partial_kernel<T, D, true, true> : decode_partial_kernel<T, D, true, false>)
+             : (aligned32 ? decode_partial_kernel<T, D, false, true> : decode_partial_kernel<T, D, false, false>);
   if (ev_b) cudaEventRecord(ev_b, st);
-  if (sparse) {
-    if (aligned32) decode_partial_kernel<T, D, true, true><<<grid, kThreads, 0, st>>>(p);
-    else decode_partial_kernel<T, D, true, false><<<grid, kThreads, 0, st>>>(p);
-  } else {
-    if (aligned32) decode_partial_kernel<T, D, false, true><<<grid, kThreads, 0, st>>>(p);
-    else decode_partial_kernel<T, D, false, false><<<grid, kThreads, 0, st>>>(p);
-  }
+  cudaError_t err = launch_pdl(kernel, grid, dim3(kThreads), st, p);
   if (ev_e) cudaEventRecord(ev_e, st);
-  if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   int launches = 1;
   if (p.n_chunks > 1) {
-    decode_merge_kernel<T, D><<<dim3((unsigned)p.H, (unsigned)B), D, 0, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+    err = launch_pdl(decode_merge_kernel<T, D>, dim3((unsigned)p.H, (unsigned)B), dim3(D), st, p);
+    if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
     ++launches;
   }
   note_launches(launches);

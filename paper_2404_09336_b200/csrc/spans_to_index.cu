@@ -34,6 +34,8 @@ spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* _
 
   const int b = blockIdx.y;
   const int tid = threadIdx.x;
+  grid_dependency_wait();
+  grid_launch_dependents();
   const int n = max(ctx_lens[b], 0);
   const int first = span_offsets[b];
   int S = span_offsets[b + 1] - first;
@@ -158,9 +160,10 @@ extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t
   if (slices > 8) slices = 8;
   const int32_t slice = (index_stride + slices - 1) / slices;
   dim3 grid((unsigned)slices, (unsigned)B);
-  ssa::spans_to_index_kernel<<<grid, ssa::kIdxThreads, 0, (cudaStream_t)stream>>>(
-      span_offsets, spans, ctx_lens, index, index_stride, slice, counts, dev_status);
-  if (cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel, grid, dim3(ssa::kIdxThreads),
+                                          (cudaStream_t)stream, span_offsets, spans, ctx_lens, index,
+                                          index_stride, slice, counts, dev_status);
+  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   ssa::note_launches(1);
   return SSA_OK;
 }

@@ -17,6 +17,29 @@ constexpr float kLn2 = 0.6931471805599453f;
 void note_launches(int n);
 void take_kernel_events(cudaEvent_t* begin, cudaEvent_t* end);
 
+// Programmatic dependent launch.  Every kernel of the library is launched
+// with the programmatic-serialization attribute: its blocks may become
+// resident while the preceding kernel of the stream is still draining, and
+// they call grid_dependency_wait() before touching any global memory, which
+// returns once that kernel has completed and its writes are visible.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
 // 16-byte read-only load that does not allocate in L1: every K/V row is used once.
