@@ -50,7 +50,7 @@ struct DecodeParams {
   uint32_t* dev_status;
   int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;
   uint32_t k_row_bytes, v_row_bytes;   // token stride of the cache in bytes
-  int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32;
+  int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32, early_release;
   float scale_log2;         // softmax scale * log2(e)
 };
 
@@ -119,6 +119,7 @@ decode_partial_kernel(const DecodeParams p) {
   const int start = chunk_id * p.chunk;
 
   grid_dependency_wait();
+  if (p.early_release) grid_launch_dependents();      // small grid: let the next kernel's blocks move in now
 
   // Everything the block needs before it can request cache rows is loaded
   // here in one go: sizes, its slice of the index list, the query row.
@@ -242,7 +243,7 @@ decode_partial_kernel(const DecodeParams p) {
 
   // all cache rows of this block have been read: the next kernel of the stream
   // may start filling the SMs this grid is leaving
-  grid_launch_dependents();
+  if (!p.early_release) grid_launch_dependents();
 
   // combine the lane groups of the block
   const int g = warp * kRowsPerLoad + sub;
@@ -396,6 +397,10 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   p.index_stride = index_stride; p.max_selected = max_selected;
   p.chunk = pl.chunk; p.n_chunks = pl.n_chunks;
   p.out_f32 = d->out_dtype == SSA_F32;
+  // A grid of a few waves releases the next kernel at once (its blocks wait on
+  // chip instead of being launched after the drain); a long grid does so only
+  // as its blocks finish, so that waiting blocks do not crowd out its own.
+  p.early_release = (long long)d->B * d->H * pl.n_chunks <= 148ll * 4 * 6;
   const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->D);
   p.scale_log2 = scale * kLog2e;
 

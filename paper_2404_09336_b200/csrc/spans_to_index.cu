@@ -34,8 +34,8 @@ spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* _
 
   const int b = blockIdx.y;
   const int tid = threadIdx.x;
-  grid_dependency_wait();
-  grid_launch_dependents();
+  grid_dependency_wait();      // dependents are released when this grid completes: blocks of a large
+                               // attention grid parked on the SMs during this kernel slowed it down
   const int n = max(ctx_lens[b], 0);
   const int first = span_offsets[b];
   int S = span_offsets[b + 1] - first;
@@ -156,8 +156,8 @@ extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t
   if (!span_offsets || !spans || !ctx_lens || !index || !counts) return SSA_ERR_NULL;
   if (B <= 0 || B > 65535 || index_stride <= 0) return SSA_ERR_SHAPE;
   if (reinterpret_cast<uintptr_t>(spans) % 8 != 0) return SSA_ERR_ALIGN;
-  int slices = (index_stride + 2047) / 2048;
-  if (slices > 8) slices = 8;
+  int slices = (index_stride + 511) / 512;           // blocks per request: 512 entries each, at most 32
+  if (slices > 32) slices = 32;
   const int32_t slice = (index_stride + slices - 1) / slices;
   dim3 grid((unsigned)slices, (unsigned)B);
   const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel, grid, dim3(ssa::kIdxThreads),
