@@ -11,7 +11,8 @@
  *
  * General conventions
  *  - Every pointer marked "dev" is a DEVICE pointer owned by the caller; the
- *    library never allocates, frees or keeps device memory between calls.
+ *    library never allocates or frees device memory, and keeps none between
+ *    calls except the fixed array named at ssa_decode_attn_sparse_noalloc.
  *    Pointers marked "host" are ordinary host pointers read during the call.
  *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
  *    the default stream).  No call synchronises or reads device memory back,
@@ -177,6 +178,43 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q,
                               const int32_t* ctx_lens, void* out, float* lse,
                               void* workspace, size_t workspace_bytes,
                               uint32_t* dev_status, void* stream);
+
+/*
+ * ssa_decode_attn_sparse for callers that cannot hand the library a
+ * workspace.  (The paper has no counterpart: its kernel runs one thread block
+ * per head and request and needs no scratch memory.)
+ *
+ * Who needs it: code that may not allocate device memory at the point of the
+ * call - a plug-in running inside a host application that owns the device
+ * allocator, a serving loop that has frozen its memory pool after start-up,
+ * or a latency-critical path where cudaMalloc (which can synchronise the whole
+ * device) is off limits.  Such a caller still passes all inputs and outputs;
+ * only the split-KV scratch comes from the library: a fixed array of
+ * SSA_STATIC_SCRATCH_BYTES bytes that lives in the library's device image, so
+ * every GPU that loads the library holds it until the process exits.
+ *
+ * Same arguments and results as ssa_decode_attn_sparse, minus the workspace.
+ * Differences:
+ *  - a request whose scratch need (what ssa_decode_workspace_bytes reports
+ *    for desc and max_selected) exceeds SSA_STATIC_SCRATCH_BYTES is rejected
+ *    with SSA_ERR_WORKSPACE and nothing is launched;
+ *  - the first call on each device looks up the array's device address (the
+ *    device must be current); make that first call outside any stream
+ *    capture.  No call allocates or frees memory;
+ *  - all calls share the one array, and it keeps whatever the previous call
+ *    left in it.  Nothing in it needs to start at zero (every slot is written
+ *    before it is read within a call), but two calls whose kernels overlap on
+ *    the GPU - different streams, or graphs launched concurrently - race on
+ *    it and corrupt each other's results.  Issue them on one stream, or order
+ *    them with events.
+ */
+#define SSA_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t ssa_decode_attn_sparse_noalloc(const ssa_attn_desc* desc, const void* q,
+                                       const void* k_cache, const void* v_cache,
+                                       const int32_t* ctx_lens, const int32_t* index,
+                                       int32_t index_stride, const int32_t* counts,
+                                       int32_t max_selected, void* out, float* lse,
+                                       uint32_t* dev_status, void* stream);
 
 /*
  * Optional timing hook for harnesses (no counterpart in the paper): the next

@@ -415,9 +415,43 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   return d->D == 128 ? launch<__half, 128>(p, d->B, sparse, a32, st) : launch<__half, 64>(p, d->B, sparse, a32, st);
 }
 
+// Scratch of ssa_decode_attn_sparse_noalloc: part of the library's device image.
+// In host code the name `g_static_scratch` is only a handle for
+// cudaGetSymbolAddress, never a device address to pass to a kernel.
+static __device__ __align__(256) unsigned char g_static_scratch[SSA_STATIC_SCRATCH_BYTES];
+
+// Device address of the array on the current device, looked up once per device.
+static void* static_scratch_address() {
+  static void* address[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!address[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+    address[dev] = ptr;
+  }
+  return address[dev];
+}
+
 }  // namespace ssa
 
 extern "C" {
+
+int32_t ssa_decode_attn_sparse_noalloc(const ssa_attn_desc* desc, const void* q, const void* k_cache,
+                                       const void* v_cache, const int32_t* ctx_lens, const int32_t* index,
+                                       int32_t index_stride, const int32_t* counts, int32_t max_selected,
+                                       void* out, float* lse, uint32_t* dev_status, void* stream) {
+  if (!desc) return SSA_ERR_NULL;
+  const int32_t rc = ssa::check_desc(desc);
+  if (rc != SSA_OK) return rc;
+  ssa::Plan pl;
+  if (max_selected <= 0 || !ssa::make_plan(desc, max_selected, &pl)) return SSA_ERR_CAPACITY;
+  if (pl.total_bytes > SSA_STATIC_SCRATCH_BYTES) return SSA_ERR_WORKSPACE;   // beyond the built-in scratch
+  void* scratch = ssa::static_scratch_address();
+  if (!scratch) return SSA_ERR_CUDA;
+  return ssa::run(desc, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out, lse,
+                  scratch, SSA_STATIC_SCRATCH_BYTES, dev_status, stream, true);
+}
 
 size_t ssa_decode_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selected) {
   ssa::Plan pl;

@@ -53,6 +53,9 @@ def _load():
     lib.ssa_decode_attn_sparse.restype = C.c_int32
     lib.ssa_decode_attn_sparse.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
                                            vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_attn_sparse_noalloc.restype = C.c_int32
+    lib.ssa_decode_attn_sparse_noalloc.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
+                                                   vp, vp, vp, vp]
     lib.ssa_decode_attn_dense.restype = C.c_int32
     lib.ssa_decode_attn_dense.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
     lib.ssa_set_kernel_events.restype = None
@@ -145,6 +148,21 @@ def decode_attn_sparse(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_s
                                     _ptr(counts), int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace),
                                     ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_sparse", rc, check)
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def decode_attn_sparse_noalloc(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_selected, out, lse=None,
+                               dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_sparse_noalloc: as decode_attn_sparse, with the scratch
+    memory taken from the library's built-in array instead of a workspace
+    tensor (for callers that must not allocate; see include/ssa.h)."""
+    rc = lib.ssa_decode_attn_sparse_noalloc(C.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens),
+                                            _ptr(index), _row_stride(index) if index is not None else 0,
+                                            _ptr(counts), int(max_selected), _ptr(out), _ptr(lse),
+                                            _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_sparse_noalloc", rc, check)
 
 
 def decode_attn_dense(desc, q, k_cache, v_cache, ctx_lens, out, lse=None, workspace=None, dev_status=None,
