@@ -177,9 +177,16 @@ def run_reference(args):
 # GPU arm
 # ---------------------------------------------------------------------------------------
 class Timer:
-    def __init__(self, torch, dist, world):
-        self.torch, self.dist, self.world = torch, dist, world
+    def __init__(self, torch, dist, world, device="cuda"):
+        self.torch, self.dist, self.world, self.device = torch, dist, world, device
         self.windows = []
+
+    def max_over_ranks(self, x):
+        if self.world > 1:
+            t = self.torch.tensor([float(x)], dtype=self.torch.float64, device=self.device)
+            self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+            return float(t.item())
+        return float(x)
 
     def sync(self):
         self.torch.cuda.synchronize()
@@ -200,16 +207,11 @@ class Timer:
         e1.record()
         self.sync()
         self.windows.append((w0, time.time()))
-        ms = e0.elapsed_time(e1)
-        if self.world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return self.max_over_ranks(e0.elapsed_time(e1))
 
     def total(self, x):
         if self.world > 1:
-            t = self.torch.tensor([float(x)], dtype=self.torch.float64, device="cuda")
+            t = self.torch.tensor([float(x)], dtype=self.torch.float64, device=self.device)
             self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM)
             return float(t.item())
         return float(x)
