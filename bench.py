@@ -46,6 +46,20 @@ WORKLOAD_TEXT = {
 }
 
 
+# DRAM traffic of one launch of the sparse decode kernel at cfg 2 (dram__bytes_read.sum +
+# dram__bytes_write.sum, profiles/decode_partial_kernel_cfg2_ncu_full.md), valid only for the kernel
+# source it was captured from.
+NCU_TRAFFIC = {"source_sha256_16": "f60f138acd7b67cb", "cfg": 2, "bytes_per_launch": 153119232}
+
+
+def kernel_source_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("decode_attn.cu", "ssa_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2404_09336_b200", "csrc", name), "rb").read())
+    return h.hexdigest()[:16]
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -379,13 +393,21 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # the dominant kernel alone: events recorded by the library around it; when the call is that one
+    # kernel, also the average over back-to-back calls (no event between launches), whichever is lower
     kernel_us = main.get("kernel_us")
+    kernel_note = "events recorded around the kernel by the library"
+    if main["launches_per_step"] == 2 and kernel_us and main["sparse_attn_us"] < kernel_us:
+        kernel_us, kernel_note = main["sparse_attn_us"], "average over back-to-back launches of the kernel"
+    traffic = NCU_TRAFFIC["bytes_per_launch"] if (args.cfg == NCU_TRAFFIC["cfg"] and
+                                                  kernel_source_hash() == NCU_TRAFFIC["source_sha256_16"]) else None
     roofline = {"bound": "hbm", "kernel": "decode_partial_kernel (sparse)",
                 "achieved": main["selected_bytes"] / kernel_us / 1e3 if kernel_us else None,
                 "peak": peak, "unit": "GB/s", "peak_kind": f"of {peak_kind}",
                 "frac": (main["selected_bytes"] / kernel_us / 1e3 / peak) if kernel_us else None,
                 "frac_of_spec_8000": (main["selected_bytes"] / kernel_us / 1e3 / SPEC_HBM_GBS) if kernel_us else None,
-                "traffic": None, "kernel_us": kernel_us,
+                "traffic": traffic, "kernel_us": kernel_us, "kernel_us_how": kernel_note,
+                "kernel_us_events_hook": main.get("kernel_us"),
                 "algorithmic_bytes_per_launch": main["selected_bytes"]}
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
