@@ -147,6 +147,30 @@ def test_multi_chunk_merge_and_tail_sizes():
             np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
 
 
+def test_batch_beyond_the_streamed_limit_takes_the_chunked_path():
+    # more requests than the persistent kernel keeps a prefix for: one block per chunk instead
+    B, H, T, D = 4100, 1, 600, 64
+    p = Problem(B, H, T, D, "bf16", seed=29)
+    rng = np.random.default_rng(9)
+    ctx = rng.integers(1, T + 1, size=B).tolist()
+    counts = [int(rng.integers(0, n + 1)) for n in ctx]
+    counts[0], counts[1], counts[2] = 0, ctx[1], 1
+    index = np.full((B, 608), -1, np.int32)
+    for b in range(B):
+        index[b, :counts[b]] = np.sort(rng.choice(ctx[b], counts[b], replace=False))
+    out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=600)
+    ref, ref_lse = oracle_sparse(p, ctx, index, counts)
+    assert status == 0
+    assert_parity(out, ref, False, "chunked path")
+    ok = np.isfinite(ref_lse)
+    np.testing.assert_allclose(lse[ok], ref_lse[ok], rtol=1e-5, atol=1e-5)
+    assert np.all(np.isneginf(lse[~ok]))
+    out_d, _, st_d = p.dense(ctx)
+    ref_d, _ = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, ctx, scale_of(D), "bf16")
+    assert st_d == 0
+    assert_parity(out_d, ref_d, False, "chunked dense")
+
+
 def test_full_span_equals_dense():
     B, H, T, D = 3, 2, 1500, 128
     p = Problem(B, H, T, D, "bf16", seed=11)

@@ -33,7 +33,7 @@ def _desc(B, H, D, T):
 def test_requests_beyond_the_builtin_scratch_are_refused():
     """Host-side check only: the pointers are never dereferenced because the
     size test fails first, so this also runs without a GPU."""
-    d = _desc(64, 32, 128, 8192)
+    d = _desc(8192, 32, 128, 8192)
     assert ssa.decode_workspace_bytes(d, 8192) > ssa.STATIC_SCRATCH_BYTES
     P = C.c_void_p(0x1000)
     before = ssa.launch_count()
