@@ -180,6 +180,49 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q,
                               uint32_t* dev_status, void* stream);
 
 /*
+ * One decode step of the method in one call (Sec. "Self-selected attention
+ * span", Inference: token generation restricted to the selected spans):
+ * ssa_spans_to_index followed by ssa_decode_attn_sparse on `stream`, with the
+ * same arguments, meanings and errors as those two calls.  Optionally the
+ * step's host-resident inputs are copied in first and its results copied out
+ * afterwards, on the same stream: when host_in is non-NULL, in_bytes bytes go
+ * from host_in to dev_in before the index kernel (a caller lays out query rows,
+ * context lengths, span offsets and spans back to back in one device arena and
+ * one pinned host arena, so that a single copy brings in everything that
+ * changes per step); when host_out is non-NULL, out_bytes bytes go from dev_out
+ * to host_out after the attention kernels.  Host arenas should be page-locked,
+ * otherwise the copies are not asynchronous.  The call does not wait for any of
+ * this work.  The KV cache is resident state and is never copied.
+ * Errors: SSA_ERR_NULL for a NULL desc/step or an inconsistent copy request,
+ * otherwise those of the two calls; nothing after a failing stage is enqueued.
+ */
+typedef struct {
+  const int32_t* span_offsets;  /* dev [B+1]                                   */
+  const int32_t* spans;         /* dev (start, end) pairs                      */
+  const int32_t* ctx_lens;      /* dev [B]                                     */
+  int32_t* index;               /* dev [B * index_stride]  (written)           */
+  int32_t* counts;              /* dev [B]                 (written)           */
+  const void* q;                /* dev                                         */
+  const void* k_cache;          /* dev                                         */
+  const void* v_cache;          /* dev                                         */
+  void* out;                    /* dev                     (written)           */
+  float* lse;                   /* dev [B*H] or NULL       (written)           */
+  void* workspace;              /* dev                                         */
+  size_t workspace_bytes;
+  uint32_t* dev_status;         /* dev [1] or NULL                             */
+  int32_t index_stride;
+  int32_t max_selected;
+  const void* host_in;          /* host (pinned) or NULL                       */
+  void* dev_in;                 /* dev                                         */
+  size_t in_bytes;
+  void* host_out;               /* host (pinned) or NULL                       */
+  const void* dev_out;          /* dev                                         */
+  size_t out_bytes;
+} ssa_step;
+
+int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* step, void* stream);
+
+/*
  * ssa_decode_attn_sparse for callers that cannot hand the library a
  * workspace.  (The paper has no counterpart: its kernel runs one thread block
  * per head and request and needs no scratch memory.)

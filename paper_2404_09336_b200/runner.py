@@ -137,16 +137,23 @@ class DecodeStep:
         context lengths, span lists) and a pinned landing buffer for what the
         caller reads back (output rows, lse, counts, status word).
         Returns (host-to-device bytes, device-to-host bytes) per step."""
+        self._host_steps = {}
         self.h_in = self.in_arena.cpu().pin_memory()
         self.h_out = torch.empty(self.out_arena.shape, dtype=torch.uint8).pin_memory()
         return self.h_in.numel(), self.h_out.numel()
 
     def step_from_host(self, stream=None):
         """Decode step whose per-step inputs start in pinned host memory and
-        whose result ends there; the KV cache is the resident state."""
-        self.in_arena.copy_(self.h_in, non_blocking=True)
-        self.step(stream)
-        self.h_out.copy_(self.out_arena, non_blocking=True)
+        whose result ends there (ssa_decode_step with both copies); the KV
+        cache is the resident state."""
+        key = (self.k.data_ptr(), self.max_selected)
+        st = self._host_steps.get(key)
+        if st is None:
+            st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q,
+                               self.k, self.v, self.max_selected, self.out, self.lse, self.workspace, self.status,
+                               host_in=self.h_in, dev_in=self.in_arena, host_out=self.h_out, dev_out=self.out_arena)
+            self._host_steps[key] = st
+        return ssa.decode_step(self.desc, st, stream)
 
     def set_spans(self, wl: Workload):
         """Replace the span lists (same geometry, same cache)."""

@@ -34,6 +34,19 @@ class AttnDesc(C.Structure):
     ]
 
 
+class Step(C.Structure):
+    """ssa_step: the arguments of one decode step (see include/ssa.h)."""
+    _fields_ = [
+        ("span_offsets", C.c_void_p), ("spans", C.c_void_p), ("ctx_lens", C.c_void_p),
+        ("index", C.c_void_p), ("counts", C.c_void_p),
+        ("q", C.c_void_p), ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("out", C.c_void_p), ("lse", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("dev_status", C.c_void_p), ("index_stride", C.c_int32), ("max_selected", C.c_int32),
+        ("host_in", C.c_void_p), ("dev_in", C.c_void_p), ("in_bytes", C.c_size_t),
+        ("host_out", C.c_void_p), ("dev_out", C.c_void_p), ("out_bytes", C.c_size_t),
+    ]
+
+
 class SsaError(RuntimeError):
     def __init__(self, fn, code):
         self.code = code
@@ -53,6 +66,8 @@ def _load():
     lib.ssa_decode_attn_sparse.restype = C.c_int32
     lib.ssa_decode_attn_sparse.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
                                            vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_step.restype = C.c_int32
+    lib.ssa_decode_step.argtypes = [C.POINTER(AttnDesc), C.POINTER(Step), vp]
     lib.ssa_decode_attn_sparse_noalloc.restype = C.c_int32
     lib.ssa_decode_attn_sparse_noalloc.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
                                                    vp, vp, vp, vp]
@@ -148,6 +163,27 @@ def decode_attn_sparse(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_s
                                     _ptr(counts), int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace),
                                     ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_sparse", rc, check)
+
+
+def make_step(span_offsets, spans, ctx_lens, index, counts, q, k_cache, v_cache, max_selected, out, lse=None,
+              workspace=None, dev_status=None, host_in=None, dev_in=None, host_out=None, dev_out=None) -> Step:
+    """Fill an ssa_step from tensors (addresses only; keep the tensors alive)."""
+    addr = lambda t: None if t is None else t.data_ptr()
+    nbytes = lambda t: 0 if t is None else t.numel() * t.element_size()
+    s = Step()
+    s.span_offsets, s.spans, s.ctx_lens = addr(span_offsets), addr(spans), addr(ctx_lens)
+    s.index, s.counts = addr(index), addr(counts)
+    s.q, s.k_cache, s.v_cache = addr(q), addr(k_cache), addr(v_cache)
+    s.out, s.lse, s.workspace, s.workspace_bytes = addr(out), addr(lse), addr(workspace), nbytes(workspace)
+    s.dev_status, s.index_stride, s.max_selected = addr(dev_status), _row_stride(index), int(max_selected)
+    s.host_in, s.dev_in, s.in_bytes = addr(host_in), addr(dev_in), nbytes(host_in)
+    s.host_out, s.dev_out, s.out_bytes = addr(host_out), addr(dev_out), nbytes(host_out)
+    return s
+
+
+def decode_step(desc: AttnDesc, step: Step, stream=None, check=True):
+    """ssa_decode_step: [copy in] -> spans_to_index -> decode_attn_sparse -> [copy out], one call."""
+    return _check("ssa_decode_step", lib.ssa_decode_step(C.byref(desc), C.byref(step), _stream(stream)), check)
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -147,8 +147,8 @@ def test_multi_chunk_merge_and_tail_sizes():
             np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
 
 
-def test_batch_beyond_the_streamed_limit_takes_the_chunked_path():
-    # more requests than the persistent kernel keeps a prefix for: one block per chunk instead
+def test_large_batch_of_short_ragged_requests():
+    # thousands of requests, one head each, lengths 0..600: several chunks per request, many empty ones
     B, H, T, D = 4100, 1, 600, 64
     p = Problem(B, H, T, D, "bf16", seed=29)
     rng = np.random.default_rng(9)
@@ -161,14 +161,14 @@ def test_batch_beyond_the_streamed_limit_takes_the_chunked_path():
     out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=600)
     ref, ref_lse = oracle_sparse(p, ctx, index, counts)
     assert status == 0
-    assert_parity(out, ref, False, "chunked path")
+    assert_parity(out, ref, False, "large batch")
     ok = np.isfinite(ref_lse)
     np.testing.assert_allclose(lse[ok], ref_lse[ok], rtol=1e-5, atol=1e-5)
     assert np.all(np.isneginf(lse[~ok]))
     out_d, _, st_d = p.dense(ctx)
     ref_d, _ = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, ctx, scale_of(D), "bf16")
     assert st_d == 0
-    assert_parity(out_d, ref_d, False, "chunked dense")
+    assert_parity(out_d, ref_d, False, "large batch dense")
 
 
 def test_full_span_equals_dense():
@@ -260,3 +260,33 @@ def test_strided_views_and_launch_counter():
     assert ssa.launch_count() > before
     ref, _ = oracle_sparse(p, [128, 128], index, [64, 64])
     assert_parity(out, ref, False, "strided q")
+
+
+def test_decode_step_in_one_call_with_host_copies():
+    # ssa_decode_step: copy in, index, attention, copy out - against the two separate calls
+    wl = inputs.make_config(2, B=5, H=4)
+    ds = DecodeStep(wl, out_dtype=torch.float32)
+    ds.step()
+    torch.cuda.synchronize()
+    want_out, want_lse = ds.out.clone(), ds.lse.clone()
+    want_counts = ds.counts.clone()
+    ds.make_host_buffers()
+    ds.in_arena.zero_()                                        # the device copy of the inputs is wiped:
+    ds.out_arena.fill_(7)                                      # everything must come from the host arena
+    ds.index.fill_(-7)
+    ds.status.zero_()
+    before = ssa.launch_count()
+    ds.step_from_host()
+    torch.cuda.synchronize()
+    assert ssa.launch_count() - before >= 2
+    assert torch.equal(ds.out, want_out) and torch.equal(ds.lse, want_lse) and torch.equal(ds.counts, want_counts)
+    host = ds.h_out.clone()
+    assert torch.equal(host, ds.out_arena.cpu())               # results landed in the pinned arena
+    assert int(ds.status.item()) == 0
+    # argument checks of the composite call
+    st = ssa.make_step(ds.span_offsets, ds.spans, ds.ctx_lens, ds.index, ds.counts, ds.q, ds.k, ds.v,
+                       ds.max_selected, ds.out, ds.lse, ds.workspace, ds.status, host_in=ds.h_in, dev_in=None)
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_NULL
+    st = ssa.make_step(ds.span_offsets, ds.spans, ds.ctx_lens, ds.index, ds.counts, ds.q, ds.k, ds.v,
+                       ds.max_selected, ds.out, ds.lse, None, ds.status)
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_WORKSPACE
