@@ -23,6 +23,11 @@ What is stated here, and where the paper defines it:
 * ``attn_alg1_blocked``   Algorithm 1 (blocked span encoding: block index +
                           block bitmask, empty blocks omitted) with the
                           readings listed below.
+* ``spans_to_blockmask``  the paper's blocked span encoding (Sec. "CUDA Kernel
+                          Design", Attention span encoding): block index and
+                          block bitmask of every block of ``bs`` positions that
+                          holds a selected position, empty blocks omitted;
+                          ``blockmask_to_index`` is its decoding.
 * ``merge_partials``      recombination of (max, sum, accumulator) partial
                           results of disjoint subsets; not in the paper (its
                           kernel runs one thread block per head and request),
@@ -227,6 +232,55 @@ def attn_alg1_blocked(q, K, V, n: int, metadata, bs: int, scale: float):
     return o, float(zmax + np.log(np.sum(E)))
 
 
+def spans_to_blockmask(spans, n: int, bs: int):
+    """Blocked encoding of the positions selected by ``spans`` in a context of
+    ``n`` rows: (block_idx int32[nb] ascending, words uint32[nb, bs // 32]).
+    Bit ``i`` of word ``w`` of a block stands for position
+    ``block * bs + 32 * w + i``."""
+    if bs % 32 != 0 or bs <= 0:
+        raise ValueError("block size must be a positive multiple of 32")
+    meta = encode_blocked(spans_to_index(spans, n), bs)
+    block_idx = np.array([blk for blk, _ in meta], dtype=np.int32)
+    words = np.zeros((len(meta), bs // 32), dtype=np.uint32)
+    for r, (_, bm) in enumerate(meta):
+        for i in np.flatnonzero(bm):
+            words[r, i // 32] |= np.uint32(1) << np.uint32(i % 32)
+    return block_idx, words
+
+
+def blockmask_to_index(block_idx, words, bs: int) -> np.ndarray:
+    """Positions named by a blocked encoding, in the order of the list."""
+    out = []
+    for blk, row in zip(np.asarray(block_idx, dtype=np.int64), np.asarray(words, dtype=np.uint32)):
+        for w, word in enumerate(row):
+            for i in range(32):
+                if (int(word) >> i) & 1:
+                    out.append(int(blk) * bs + 32 * w + i)
+    return np.asarray(out, dtype=np.int32)
+
+
+def spans_to_blockmask_batch(span_offsets, spans, ctx_lens, bs: int, block_stride: int):
+    """Batch form in the library's padded layout: block_idx[B, block_stride]
+    (-1 past the count), words[B, block_stride, bs // 32], counts[B], status
+    bits.  A request with more than ``block_stride`` blocks keeps the first."""
+    span_offsets = np.asarray(span_offsets, dtype=np.int64)
+    spans = np.asarray(spans, dtype=np.int64).reshape(-1, 2)
+    B = len(ctx_lens)
+    block_idx = np.full((B, block_stride), -1, dtype=np.int32)
+    words = np.zeros((B, block_stride, bs // 32), dtype=np.uint32)
+    counts = np.zeros(B, dtype=np.int32)
+    status = 0
+    for b in range(B):
+        sp = spans[span_offsets[b]:span_offsets[b + 1]]
+        status |= spans_status(sp, int(ctx_lens[b]))
+        bi, wd = spans_to_blockmask(sp, int(ctx_lens[b]), bs)
+        if len(bi) > block_stride:
+            status |= ST_OVERFLOW
+        c = min(len(bi), block_stride)
+        block_idx[b, :c], words[b, :c], counts[b] = bi[:c], wd[:c], c
+    return block_idx, words, counts, status
+
+
 def merge_partials(ms, ls, accs):
     """Combine partial results of disjoint position subsets:
     m = max m_k, l = sum l_k e^(m_k - m), out = sum acc_k e^(m_k - m) / l."""
@@ -278,6 +332,21 @@ def decode_attn_sparse(q, k_cache, v_cache, ctx_lens, index, counts, scale,
             out[b, h] = o
             lse[b, h] = e
     return out, lse
+
+
+def decode_attn_blockmask(q, k_cache, v_cache, ctx_lens, block_idx, words, counts, bs: int, scale,
+                          dtype: str = "bf16", heads=None, seqs=None):
+    """Span-restricted decode attention from the blocked encoding: the
+    positions it names (those inside the context) are attended.  Same
+    conventions as ``decode_attn_sparse``."""
+    B = q.shape[0]
+    stride = max(int(np.max(counts)) * bs if B else 0, 1)
+    index = np.full((B, stride), -1, dtype=np.int32)
+    cnt = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        pos = blockmask_to_index(block_idx[b][: int(counts[b])], words[b][: int(counts[b])], bs)
+        index[b, : len(pos)], cnt[b] = pos, len(pos)
+    return decode_attn_sparse(q, k_cache, v_cache, ctx_lens, index, cnt, scale, dtype, heads, seqs)
 
 
 def decode_attn_dense(q, k_cache, v_cache, ctx_lens, scale,
