@@ -180,6 +180,52 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q,
                               uint32_t* dev_status, void* stream);
 
 /*
+ * The paper's own metadata format (Sec. "CUDA Kernel Design", Attention span
+ * encoding): the context is cut into blocks of `block_size` positions; for
+ * every block that holds at least one selected position the list records the
+ * block index and a bitmask of the selected positions inside it; blocks
+ * without selected positions are omitted; every request has its own list.
+ *
+ * ssa_spans_to_blockmask builds it from span lists (same span semantics and
+ * status bits as ssa_spans_to_index):
+ *   block_idx  [b*block_stride + 0 .. block_counts[b])  ascending block indices
+ *   block_mask [(b*block_stride + r) * (block_size/32) + w]  32-bit words of
+ *              list entry r; bit i of word w stands for position
+ *              block_idx*block_size + 32*w + i
+ * Entries past block_counts[b] are left untouched; more than block_stride
+ * blocks keep the first block_stride (SSA_DEV_OVERFLOW).
+ * block_size in {32, 64, 128, 256}.  All pointers dev; span_offsets, spans,
+ * ctx_lens as in ssa_spans_to_index.
+ * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE, SSA_ERR_UNSUPPORTED (block_size),
+ * SSA_ERR_ALIGN, SSA_ERR_CUDA.
+ */
+int32_t ssa_spans_to_blockmask(const int32_t* span_offsets, const int32_t* spans,
+                               const int32_t* ctx_lens, int32_t B, int32_t block_size,
+                               int32_t* block_idx, uint32_t* block_mask, int32_t block_stride,
+                               int32_t* block_counts, uint32_t* dev_status, void* stream);
+
+/*
+ * Span-restricted decode attention from that format (Algorithm 1): same
+ * result, options and errors as ssa_decode_attn_sparse, with the attended set
+ * of request b given by its first block_counts[b] list entries.  Only the rows
+ * whose bit is set are read (the bitmask is expanded on chip; a partially
+ * selected block costs its selected rows, not the whole block).  Bits naming
+ * positions outside [0, ctx_lens[b]) are skipped (SSA_DEV_BAD_INDEX); a block
+ * listed twice counts twice.  `max_blocks` is a host-side upper bound on every
+ * block_counts[b] (1 <= max_blocks <= block_stride); larger counts are clamped
+ * (SSA_DEV_BAD_COUNT).  Workspace: ssa_decode_blockmask_workspace_bytes.
+ */
+size_t ssa_decode_blockmask_workspace_bytes(const ssa_attn_desc* desc, int32_t block_size,
+                                            int32_t max_blocks);
+int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, const void* k_cache,
+                                  const void* v_cache, const int32_t* ctx_lens,
+                                  const int32_t* block_idx, const uint32_t* block_mask,
+                                  int32_t block_stride, const int32_t* block_counts,
+                                  int32_t block_size, int32_t max_blocks, void* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                  void* stream);
+
+/*
  * One decode step of the method in one call (Sec. "Self-selected attention
  * span", Inference: token generation restricted to the selected spans):
  * ssa_spans_to_index followed by ssa_decode_attn_sparse on `stream`, with the
