@@ -16,6 +16,11 @@
 // block normalises and stores the output itself; otherwise it stores the
 // unnormalised triple to the workspace and
 // Pass 2 (decode_merge_kernel) combines the chunks of one (request, head).
+//
+// The attended rows of a block come from one of three sources (kMode): every
+// position (dense), a slice of the request's index list, or a run of entries
+// of the request's blocked (block index, bitmask) list, whose set bits the
+// block expands into positions in shared memory before reading any row.
 #include "ssa_common.cuh"
 
 namespace ssa {
@@ -35,6 +40,8 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kU = SSA_U;              // 32-byte loads in flight per lane, per tensor
 constexpr int kMaxChunk = 512;         // index entries staged per block
 constexpr int kIdxPerThread = kMaxChunk / kThreads;
+constexpr int kMaskChunk = 256;        // positions a block expands from bitmasks
+enum { kDense = 0, kIndex = 1, kBlockMask = 2 };
 
 struct DecodeParams {
   const void* q;
@@ -42,7 +49,10 @@ struct DecodeParams {
   const void* v;
   const int32_t* ctx_lens;
   const int32_t* index;     // sparse only
-  const int32_t* counts;    // sparse only (NULL selects the dense count)
+  const int32_t* counts;    // list lengths: index entries or listed blocks (NULL selects the dense count)
+  const int32_t* block_idx; // blocked list only
+  const uint32_t* block_mask;
+  int32_t block_size, block_stride;
   void* out;
   float* lse;
   float* ws_acc;            // [B*H*n_chunks, D]
@@ -99,9 +109,10 @@ __device__ __forceinline__ void zero_piece(Piece& r) {
   for (int i = 0; i < 8; ++i) r.w[i] = 0u;
 }
 
-template <typename T, int D, bool kSparse, bool kAligned32>
+template <typename T, int D, int kMode, bool kAligned32>
 __global__ void __launch_bounds__(kThreads, SSA_MIN_BLOCKS)
 decode_partial_kernel(const DecodeParams p) {
+  constexpr bool kSparse = kMode != kDense;           // positions come from shared memory
   constexpr int kLanesPerRow = D / 16;                // 32-byte pieces per row
   constexpr int kRowsPerLoad = 32 / kLanesPerRow;     // rows one warp-wide load covers
   constexpr int kTileRows = kRowsPerLoad * kU;        // rows per warp per iteration
@@ -112,6 +123,7 @@ decode_partial_kernel(const DecodeParams p) {
   __shared__ __align__(16) float s_acc[kGroups][D];
   __shared__ float s_m[kGroups], s_l[kGroups];
   __shared__ int s_bad;
+  __shared__ int s_wcount[kWarps];
 
   const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -124,7 +136,7 @@ decode_partial_kernel(const DecodeParams p) {
   // Everything the block needs before it can request cache rows is loaded
   // here in one go: sizes, its slice of the index list, the query row.
   int32_t raw[kIdxPerThread];
-  if (kSparse) {
+  if (kMode == kIndex) {
     const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
 #pragma unroll
     for (int j = 0; j < kIdxPerThread; ++j) {
@@ -141,9 +153,41 @@ decode_partial_kernel(const DecodeParams p) {
   int n, c;
   request_sizes(p, b, n, c, flags);
   if (start >= c && chunk_id > 0) return;             // chunk 0 always reports
-  const int cnt = max(0, min(p.chunk, c - start));
+  int cnt = max(0, min(p.chunk, c - start));          // list entries of this block; rows, except for bitmasks
 
-  if (kSparse) {
+  if (kMode == kBlockMask) {
+    // expand the set bits of up to p.chunk listed blocks into positions, in list order
+    const int wpb = p.block_size / 32;
+    const int64_t entry0 = (int64_t)b * p.block_stride + start;
+    int rows = 0;
+    for (int base = 0; base < kMaskChunk; base += kThreads) {
+      const int i = base + tid, r = i / p.block_size, bit = i % p.block_size;
+      int pos = -1;
+      if (r < cnt) {
+        const int blk = __ldg(p.block_idx + entry0 + r);
+        const uint32_t word = __ldg(p.block_mask + (entry0 + r) * wpb + (bit >> 5));
+        if ((word >> (bit & 31)) & 1u) {
+          if (blk >= 0 && blk <= (n - 1) / p.block_size && blk * p.block_size + bit < n)
+            pos = blk * p.block_size + bit;
+          else
+            flags |= SSA_DEV_BAD_INDEX;
+        }
+      }
+      const uint32_t ballot = __ballot_sync(0xffffffffu, pos >= 0);
+      if (lane == 0) s_wcount[warp] = __popc(ballot);
+      __syncthreads();
+      int at = rows + __popc(ballot & ((1u << lane) - 1u));
+#pragma unroll
+      for (int k = 0; k < kWarps; ++k) {
+        if (k < warp) at += s_wcount[k];
+        rows += s_wcount[k];
+      }
+      if (pos >= 0) s_idx[at] = pos;
+      __syncthreads();
+    }
+    cnt = rows;
+  }
+  if (kMode == kIndex) {
     __syncthreads();                                  // s_bad cleared
 #pragma unroll
     for (int j = 0; j < kIdxPerThread; ++j) {
@@ -160,7 +204,7 @@ decode_partial_kernel(const DecodeParams p) {
     const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
     if (f) atomicOr(p.dev_status, f);
   }
-  const bool any_bad = kSparse ? (s_bad != 0) : false;
+  const bool any_bad = kMode == kIndex ? (s_bad != 0) : false;
 
   const char* kbase = reinterpret_cast<const char*>(
       reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)h * p.k_sh + col * 16);
@@ -320,6 +364,19 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   return true;
 }
 
+// Blocked lists: a block of the grid expands as many list entries as fit kMaskChunk positions.
+static bool make_plan_blockmask(const ssa_attn_desc* d, int block_size, int max_blocks, Plan* pl) {
+  if (!d || d->B <= 0 || d->H <= 0 || max_blocks <= 0) return false;
+  if (d->D != 64 && d->D != 128) return false;
+  if (block_size != 32 && block_size != 64 && block_size != 128 && block_size != 256) return false;
+  const long long units = (long long)d->B * d->H;
+  pl->chunk = kMaskChunk / block_size;
+  pl->n_chunks = (max_blocks + pl->chunk - 1) / pl->chunk;
+  pl->acc_bytes = ((size_t)units * pl->n_chunks * d->D * sizeof(float) + 255) / 256 * 256;
+  pl->total_bytes = pl->acc_bytes + ((size_t)units * pl->n_chunks * sizeof(float2) + 255) / 256 * 256;
+  return true;
+}
+
 static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
 static int32_t check_desc(const ssa_attn_desc* d) {
@@ -339,13 +396,17 @@ static int32_t check_desc(const ssa_attn_desc* d) {
 }
 
 template <typename T, int D>
-static int32_t launch(const DecodeParams& p, int B, bool sparse, bool aligned32, cudaStream_t st) {
+static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cudaStream_t st) {
   cudaEvent_t ev_b, ev_e;
   take_kernel_events(&ev_b, &ev_e);
   dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
-  void (*kernel)(const DecodeParams) =
-      sparse ? (aligned32 ? decode_partial_kernel<T, D, true, true> : decode_partial_kernel<T, D, true, false>)
-             : (aligned32 ? decode_partial_kernel<T, D, false, true> : decode_partial_kernel<T, D, false, false>);
+  void (*kernel)(const DecodeParams);
+  if (mode == kIndex)
+    kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true> : decode_partial_kernel<T, D, kIndex, false>;
+  else if (mode == kBlockMask)
+    kernel = aligned32 ? decode_partial_kernel<T, D, kBlockMask, true> : decode_partial_kernel<T, D, kBlockMask, false>;
+  else
+    kernel = aligned32 ? decode_partial_kernel<T, D, kDense, true> : decode_partial_kernel<T, D, kDense, false>;
   if (ev_b) cudaEventRecord(ev_b, st);
   cudaError_t err = launch_pdl(kernel, grid, dim3(kThreads), st, p);
   if (ev_e) cudaEventRecord(ev_e, st);
@@ -360,29 +421,48 @@ static int32_t launch(const DecodeParams& p, int B, bool sparse, bool aligned32,
   return SSA_OK;
 }
 
+// A request's attended set in the blocked encoding (mode kBlockMask).
+struct BlockList { const int32_t* block_idx; const uint32_t* block_mask; int32_t block_size; };
+
+// mode kDense: index/counts unused.  kIndex: the index list.  kBlockMask: `counts`
+// are the numbers of listed blocks, `index_stride` the list capacity in blocks,
+// `max_selected` the host bound on listed blocks, `bl` the lists.
 static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const void* v,
                    const int32_t* ctx_lens, const int32_t* index, int32_t index_stride,
                    const int32_t* counts, int32_t max_selected, void* out, float* lse,
-                   void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream, bool sparse) {
+                   void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream, int mode,
+                   const BlockList* bl = nullptr) {
+  const bool sparse = mode == kIndex;
   if (!d || !q || !k || !v || !ctx_lens || !out) return SSA_ERR_NULL;
   if (sparse && (!index || !counts)) return SSA_ERR_NULL;
+  if (mode == kBlockMask && (!bl || !bl->block_idx || !bl->block_mask || !counts)) return SSA_ERR_NULL;
   const int32_t rc = check_desc(d);
   if (rc != SSA_OK) return rc;
-  if (sparse) {
+  if (mode != kDense) {
     if (index_stride <= 0 || max_selected <= 0 || max_selected > index_stride) return SSA_ERR_CAPACITY;
   } else {
     max_selected = d->max_ctx;
   }
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(ws)) return SSA_ERR_ALIGN;
   Plan pl;
-  if (!make_plan(d, max_selected, &pl)) return SSA_ERR_SHAPE;
+  if (mode == kBlockMask) {
+    if (bl->block_size != 32 && bl->block_size != 64 && bl->block_size != 128 && bl->block_size != 256)
+      return SSA_ERR_UNSUPPORTED;
+    if (!make_plan_blockmask(d, bl->block_size, max_selected, &pl)) return SSA_ERR_SHAPE;
+  } else if (!make_plan(d, max_selected, &pl)) {
+    return SSA_ERR_SHAPE;
+  }
   if (!ws || ws_bytes < pl.total_bytes) return SSA_ERR_WORKSPACE;
 
   DecodeParams p;
   p.q = q; p.k = k; p.v = v;
   p.ctx_lens = ctx_lens;
   p.index = sparse ? index : nullptr;
-  p.counts = sparse ? counts : nullptr;
+  p.counts = mode != kDense ? counts : nullptr;
+  p.block_idx = mode == kBlockMask ? bl->block_idx : nullptr;
+  p.block_mask = mode == kBlockMask ? bl->block_mask : nullptr;
+  p.block_size = mode == kBlockMask ? bl->block_size : 0;
+  p.block_stride = mode == kBlockMask ? index_stride : 0;
   p.out = out; p.lse = lse;
   p.ws_acc = reinterpret_cast<float*>(ws);
   p.ws_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(ws) + pl.acc_bytes);
@@ -410,9 +490,9 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
                    d->v_stride_b % 16 == 0 && d->v_stride_t % 16 == 0 && d->v_stride_h % 16 == 0;
   cudaStream_t st = (cudaStream_t)stream;
   if (d->kv_dtype == SSA_BF16)
-    return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, sparse, a32, st)
-                       : launch<__nv_bfloat16, 64>(p, d->B, sparse, a32, st);
-  return d->D == 128 ? launch<__half, 128>(p, d->B, sparse, a32, st) : launch<__half, 64>(p, d->B, sparse, a32, st);
+    return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, mode, a32, st)
+                       : launch<__nv_bfloat16, 64>(p, d->B, mode, a32, st);
+  return d->D == 128 ? launch<__half, 128>(p, d->B, mode, a32, st) : launch<__half, 64>(p, d->B, mode, a32, st);
 }
 
 // Scratch of ssa_decode_attn_sparse_noalloc: part of the library's device image.
@@ -450,7 +530,24 @@ int32_t ssa_decode_attn_sparse_noalloc(const ssa_attn_desc* desc, const void* q,
   void* scratch = ssa::static_scratch_address();
   if (!scratch) return SSA_ERR_CUDA;
   return ssa::run(desc, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out, lse,
-                  scratch, SSA_STATIC_SCRATCH_BYTES, dev_status, stream, true);
+                  scratch, SSA_STATIC_SCRATCH_BYTES, dev_status, stream, ssa::kIndex);
+}
+
+size_t ssa_decode_blockmask_workspace_bytes(const ssa_attn_desc* desc, int32_t block_size, int32_t max_blocks) {
+  ssa::Plan pl;
+  if (!desc || ssa::check_desc(desc) != SSA_OK || !ssa::make_plan_blockmask(desc, block_size, max_blocks, &pl))
+    return 0;
+  return pl.total_bytes;
+}
+
+int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, const void* k_cache,
+                                  const void* v_cache, const int32_t* ctx_lens, const int32_t* block_idx,
+                                  const uint32_t* block_mask, int32_t block_stride, const int32_t* block_counts,
+                                  int32_t block_size, int32_t max_blocks, void* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream) {
+  const ssa::BlockList bl = {block_idx, block_mask, block_size};
+  return ssa::run(desc, q, k_cache, v_cache, ctx_lens, nullptr, block_stride, block_counts, max_blocks, out, lse,
+                  workspace, workspace_bytes, dev_status, stream, ssa::kBlockMask, &bl);
 }
 
 size_t ssa_decode_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selected) {
@@ -465,7 +562,7 @@ int32_t ssa_decode_attn_sparse(const ssa_attn_desc* desc, const void* q, const v
                                void* out, float* lse, void* workspace, size_t workspace_bytes,
                                uint32_t* dev_status, void* stream) {
   return ssa::run(desc, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out,
-                  lse, workspace, workspace_bytes, dev_status, stream, true);
+                  lse, workspace, workspace_bytes, dev_status, stream, ssa::kIndex);
 }
 
 int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q, const void* k_cache,
@@ -473,7 +570,7 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q, const vo
                               void* workspace, size_t workspace_bytes, uint32_t* dev_status,
                               void* stream) {
   return ssa::run(desc, q, k_cache, v_cache, ctx_lens, nullptr, 0, nullptr, 0, out, lse, workspace,
-                  workspace_bytes, dev_status, stream, false);
+                  workspace_bytes, dev_status, stream, ssa::kDense);
 }
 
 }  // extern "C"
