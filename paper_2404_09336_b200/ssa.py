@@ -66,6 +66,13 @@ def _load():
     lib.ssa_decode_attn_sparse.restype = C.c_int32
     lib.ssa_decode_attn_sparse.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
                                            vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_spans_to_blockmask.restype = C.c_int32
+    lib.ssa_spans_to_blockmask.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp, vp, C.c_int32, vp, vp, vp]
+    lib.ssa_decode_blockmask_workspace_bytes.restype = C.c_size_t
+    lib.ssa_decode_blockmask_workspace_bytes.argtypes = [C.POINTER(AttnDesc), C.c_int32, C.c_int32]
+    lib.ssa_decode_attn_blockmask.restype = C.c_int32
+    lib.ssa_decode_attn_blockmask.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
+                                              C.c_int32, vp, vp, vp, C.c_size_t, vp, vp]
     lib.ssa_decode_step.restype = C.c_int32
     lib.ssa_decode_step.argtypes = [C.POINTER(AttnDesc), C.POINTER(Step), vp]
     lib.ssa_decode_attn_sparse_noalloc.restype = C.c_int32
@@ -163,6 +170,32 @@ def decode_attn_sparse(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_s
                                     _ptr(counts), int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace),
                                     ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_sparse", rc, check)
+
+
+def spans_to_blockmask(span_offsets, spans, ctx_lens, block_size, block_idx, block_mask, block_counts,
+                       dev_status=None, stream=None, check=True):
+    """ssa_spans_to_blockmask: block_idx[B, stride], block_mask[B, stride, block_size/32] and
+    block_counts[B] are written."""
+    rc = lib.ssa_spans_to_blockmask(_ptr(span_offsets), _ptr(spans), _ptr(ctx_lens), int(ctx_lens.numel()),
+                                    int(block_size), _ptr(block_idx), _ptr(block_mask), _row_stride(block_idx),
+                                    _ptr(block_counts), _ptr(dev_status), _stream(stream))
+    return _check("ssa_spans_to_blockmask", rc, check)
+
+
+def decode_blockmask_workspace_bytes(desc: AttnDesc, block_size: int, max_blocks: int) -> int:
+    return int(lib.ssa_decode_blockmask_workspace_bytes(C.byref(desc), int(block_size), int(max_blocks)))
+
+
+def decode_attn_blockmask(desc, q, k_cache, v_cache, ctx_lens, block_idx, block_mask, block_counts, block_size,
+                          max_blocks, out, lse=None, workspace=None, dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_blockmask: out (and lse) are written."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_blockmask(C.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens),
+                                       _ptr(block_idx), _ptr(block_mask),
+                                       _row_stride(block_idx) if block_idx is not None else 0, _ptr(block_counts),
+                                       int(block_size), int(max_blocks), _ptr(out), _ptr(lse), _ptr(workspace),
+                                       ws_bytes, _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_blockmask", rc, check)
 
 
 def make_step(span_offsets, spans, ctx_lens, index, counts, q, k_cache, v_cache, max_selected, out, lse=None,
