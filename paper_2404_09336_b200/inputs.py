@@ -226,3 +226,25 @@ def make_config(cfg: int, density: float | None = None, B: int | None = None, H:
     else:
         raise ValueError(f"no workload {cfg}")
     return _finish(name, seed, B, H, D, T, dtype, ctx, per_seq, first_id)
+
+
+def make_microbench(ctx: int, sparsity_block: int, B: int = 64, H: int = 32, max_ctx: int | None = None,
+                    first_id: int = 0) -> Workload:
+    """The paper's kernel micro-benchmark (Sec. "Custom CUDA kernel
+    benchmarking"): one new token over ``ctx`` preceding tokens of which half
+    are ignored; the binary mask is made of blocks of ones of size
+    ``sparsity_block`` (exactly half of the aligned blocks, drawn at random
+    per request); batch 64; LLaMA-7B heads.  ``max_ctx`` lets several context
+    lengths share one cache allocation."""
+    if ctx % sparsity_block:
+        raise ValueError("the context must be a multiple of the sparsity block")
+    seed = BASE_SEED + 6000
+    n_blocks = ctx // sparsity_block
+    per_seq = []
+    for b in range(first_id, first_id + B):
+        r = _rng(seed + ctx + sparsity_block, b, 0)
+        keep = np.sort(r.permutation(n_blocks)[: n_blocks // 2])
+        per_seq.append(_shuffled(r, [(int(k) * sparsity_block, (int(k) + 1) * sparsity_block) for k in keep]))
+    wl = _finish(f"paper_microbench_ctx{ctx}_sb{sparsity_block}", seed, B, H, 128, max_ctx or ctx, "bf16",
+                 [ctx] * B, per_seq, first_id)
+    return wl

@@ -126,6 +126,32 @@ class DecodeStep:
         return ssa.decode_attn_dense(self.desc, self.q, self.k, self.v, self.ctx_lens, self.out, self.lse,
                                      self.workspace, self.status, stream)
 
+    # ---- the paper's blocked encoding as the metadata format ---------------------------
+    def enable_blockmask(self, block_size: int = 256):
+        """Buffers for the (block index, bitmask) lists of every request."""
+        B, dev = self.wl.B, self.device
+        self.block_size = block_size
+        self.block_stride = (self.wl.max_ctx + block_size - 1) // block_size
+        self.block_idx = torch.full((B, self.block_stride), -7, dtype=torch.int32, device=dev)
+        self.block_mask = torch.zeros((B, self.block_stride, block_size // 32), dtype=torch.int32, device=dev)
+        self.block_counts = torch.zeros((B,), dtype=torch.int32, device=dev)
+        need = ssa.decode_blockmask_workspace_bytes(self.desc, block_size, self.block_stride)
+        if need > self.workspace.numel():
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+
+    def build_blockmask(self, stream=None):
+        return ssa.spans_to_blockmask(self.span_offsets, self.spans, self.ctx_lens, self.block_size, self.block_idx,
+                                      self.block_mask, self.block_counts, self.status, stream)
+
+    def attend_blockmask(self, stream=None):
+        return ssa.decode_attn_blockmask(self.desc, self.q, self.k, self.v, self.ctx_lens, self.block_idx,
+                                         self.block_mask, self.block_counts, self.block_size, self.block_stride,
+                                         self.out, self.lse, self.workspace, self.status, stream)
+
+    def step_blockmask(self, stream=None):
+        self.build_blockmask(stream)
+        self.attend_blockmask(stream)
+
     def step(self, stream=None):
         """One decode step of the method: span lists -> index lists -> attention."""
         self.build_index(stream)
