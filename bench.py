@@ -329,6 +329,50 @@ def measure(torch, ssa, timer, ds, steps, warmup, peak, kernel_pass=True):
     return res
 
 
+def paper_microbench(torch, ssa, timer, n_iter=20):
+    """The paper's kernel micro-benchmark (50 % of the preceding tokens ignored, mask made of
+    blocks of ones of a given size, batch 64, 1024..8192 preceding tokens): speedup of the
+    span-restricted step over this library's dense kernel, through the index list and through
+    the paper's blocked (index, bitmask) encoding with 256-position blocks."""
+    from paper_2404_09336_b200 import inputs
+    from paper_2404_09336_b200.runner import DecodeStep
+    T, B = 8192, 64
+    base = inputs.make_microbench(T, 256, B=B, max_ctx=T)
+    ds = DecodeStep(base, kv_copies=1, index_stride=T // 2, max_selected=T // 2, span_capacity=B * (T // 64))
+    ds.enable_blockmask(256)
+    rows = []
+    for ctx in (1024, 2048, 4096, 8192):
+        for sb in (32, 64, 128, 256):
+            ds.set_spans(inputs.make_microbench(ctx, sb, B=B, max_ctx=T))
+            for fn in (ds.step, ds.step_blockmask, ds.attend_dense):
+                fn()
+            torch.cuda.synchronize()
+            if int(ds.status.item()) != 0:
+                raise SystemExit("micro-benchmark raised a device status flag")
+            t_idx = timer.run(lambda i: ds.step(), n_iter) / n_iter * 1e3
+            t_bm = timer.run(lambda i: ds.step_blockmask(), n_iter) / n_iter * 1e3
+            t_dense = timer.run(lambda i: ds.attend_dense(), n_iter) / n_iter * 1e3
+            sel = B * (ctx // 2) * base.kv_bytes_per_token()
+            rows.append({"ctx": ctx, "sparsity_block": sb, "dense_us": round(t_dense, 2),
+                         "index_path_us": round(t_idx, 2), "blockmask_path_us": round(t_bm, 2),
+                         "speedup_index": round(t_dense / t_idx, 3), "speedup_blockmask": round(t_dense / t_bm, 3),
+                         "index_path_gbs": round(sel / t_idx / 1e3, 1)})
+    geo = lambda xs: float(np.exp(np.mean(np.log(xs))))
+    summary = {"geomean_speedup_index": round(geo([r["speedup_index"] for r in rows]), 3),
+               "geomean_speedup_blockmask": round(geo([r["speedup_blockmask"] for r in rows]), 3)}
+    for sb in (32, 64, 128, 256):
+        summary[f"geomean_speedup_index_sb{sb}"] = round(
+            geo([r["speedup_index"] for r in rows if r["sparsity_block"] == sb]), 3)
+        summary[f"geomean_speedup_blockmask_sb{sb}"] = round(
+            geo([r["speedup_blockmask"] for r in rows if r["sparsity_block"] == sb]), 3)
+    del ds
+    torch.cuda.empty_cache()
+    return {"what": "paper kernel micro-benchmark: batch 64, 32 heads x 128, 50% of tokens ignored, speedup vs "
+                    "ssa_decode_attn_dense (the paper compares with HF attention on an A100: 1.29x overall, "
+                    "0.97/1.2/1.6/1.6x at sparsity block 32/64/128/256)",
+            "summary": summary, "rows": rows}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -469,6 +513,8 @@ def run_ours(args):
         five = [r for r in sweep if r["workload"].startswith("cfg5")]
         cross = next((r["density"] for r in five if r["speedup_vs_dense"] < 1.0), None)
         line["crossover_density"] = cross
+        if args.sweep != "none":
+            line["paper_microbench"] = paper_microbench(torch, ssa, timer)
         line["cpu_baseline"] = time_oracle(args.cfg, budget_s=15.0)
         for k in ("seconds", "ms_per_step", "steps"):
             line["cpu_baseline"].pop(k, None)
