@@ -118,11 +118,12 @@ decode_partial_kernel(const DecodeParams p) {
   constexpr int kTileRows = kRowsPerLoad * kU;        // rows per warp per iteration
   constexpr int kGroups = kWarps * kRowsPerLoad;      // independent softmax streams
   static_assert(kThreads >= D, "the epilogue uses one thread per output element");
+  static_assert(kMaxChunk == kIdxPerThread * kThreads && (32 * kIdxPerThread) % kTileRows == 0,
+                "a warp stages whole tiles");
 
   __shared__ int32_t s_idx[kSparse ? kMaxChunk : 1];
   __shared__ __align__(16) float s_acc[kGroups][D];
   __shared__ float s_m[kGroups], s_l[kGroups];
-  __shared__ int s_bad;
   __shared__ int s_wcount[kWarps];
 
   const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -135,15 +136,20 @@ decode_partial_kernel(const DecodeParams p) {
 
   // Everything the block needs before it can request cache rows is loaded
   // here in one go: sizes, its slice of the index list, the query row.
+  // A warp stages exactly the list entries of its own tiles (entry i of the
+  // warp's share is row staged_row(i) of the block), so staging needs no block
+  // barrier, only a warp one.
+  auto staged_row = [&](int i) {
+    return warp * kTileRows + (i / kTileRows) * (kWarps * kTileRows) + (i % kTileRows);
+  };
   int32_t raw[kIdxPerThread];
   if (kMode == kIndex) {
     const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
 #pragma unroll
     for (int j = 0; j < kIdxPerThread; ++j) {
-      const int i = tid + j * kThreads;
-      raw[j] = (i < p.chunk && start + i < p.max_selected) ? __ldg(row + i) : -1;
+      const int r = staged_row(lane + 32 * j);
+      raw[j] = (r < p.chunk && start + r < p.max_selected) ? __ldg(row + r) : -1;
     }
-    if (tid == 0) s_bad = 0;
   }
   Piece qraw;
   load_piece<false>(qraw, reinterpret_cast<const char*>(
@@ -187,24 +193,25 @@ decode_partial_kernel(const DecodeParams p) {
     }
     cnt = rows;
   }
+  bool any_bad = false;                               // warp-uniform: an entry of this warp's tiles is out of range
   if (kMode == kIndex) {
-    __syncthreads();                                  // s_bad cleared
+    bool bad = false;
 #pragma unroll
     for (int j = 0; j < kIdxPerThread; ++j) {
-      const int i = tid + j * kThreads;
-      if (i < cnt) {
+      const int r = staged_row(lane + 32 * j);
+      if (r < cnt) {
         int v = raw[j];
-        if (v < 0 || v >= n) { v = -1; flags |= SSA_DEV_BAD_INDEX; s_bad = 1; }
-        s_idx[i] = v;
+        if (v < 0 || v >= n) { v = -1; flags |= SSA_DEV_BAD_INDEX; bad = true; }
+        s_idx[r] = v;
       }
     }
-    __syncthreads();
+    any_bad = __any_sync(0xffffffffu, bad) != 0;      // also orders the stores before the warp's reads
+    __syncwarp();
   }
   if (p.dev_status && h == 0) {
     const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
     if (f) atomicOr(p.dev_status, f);
   }
-  const bool any_bad = kMode == kIndex ? (s_bad != 0) : false;
 
   const char* kbase = reinterpret_cast<const char*>(
       reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)h * p.k_sh + col * 16);
