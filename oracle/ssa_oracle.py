@@ -28,6 +28,15 @@ What is stated here, and where the paper defines it:
                           block bitmask of every block of ``bs`` positions that
                           holds a selected position, empty blocks omitted;
                           ``blockmask_to_index`` is its decoding.
+* ``resolve_references``  anchors and references to token spans (Sec.
+                          "Self-selected attention span": anchors identify
+                          groups of contiguous tokens, the model names anchors,
+                          generation attends to the named groups; the worked
+                          examples of the arithmetic and summarization figures:
+                          "[-1]" is the previous line, the instruction is always
+                          attended, the line being generated attends to itself).
+                          The paper gives no algorithm; the rules are stated in
+                          the function.
 * ``merge_partials``      recombination of (max, sum, accumulator) partial
                           results of disjoint subsets; not in the paper (its
                           kernel runs one thread block per head and request),
@@ -62,6 +71,7 @@ import numpy as np
 ST_BAD_SPAN = 1    # start < 0 or start > end
 ST_CLIPPED = 2     # end > context length
 ST_OVERFLOW = 4    # more selected positions than the index row can hold
+ST_BAD_REF = 64    # a reference named an anchor or line that does not exist
 
 
 # --------------------------------------------------------------------------
@@ -230,6 +240,49 @@ def attn_alg1_blocked(q, K, V, n: int, metadata, bs: int, scale: float):
             if delta + i < n and A[delta + i] != 0.0:
                 o += A[delta + i] * V[delta + i]
     return o, float(zmax + np.log(np.sum(E)))
+
+
+def resolve_references(lines, anchor_line, refs, prefix_len: int, line_start: int, ctx_len: int,
+                       span_stride: int | None = None):
+    """Token spans a request attends to while it generates its current line.
+
+    ``lines``       (start, end) of the completed lines (groups) of the context,
+                    in order of appearance;
+    ``anchor_line`` anchor id -> index into ``lines`` of the line it identifies;
+    ``refs``        (lo, hi) pairs.  0 <= lo <= hi: the anchors lo..hi; lo == hi
+                    == -k (k >= 1): the k-th line before the current one, i.e.
+                    ``lines[len(lines) - k]``.
+    Result, in this order: the always-attended prefix [0, prefix_len), the
+    current line [line_start, ctx_len), then for each reference in turn one span
+    per named line.  References to anchors or lines that do not exist, and
+    pairs of any other form, are skipped and flagged.  With ``span_stride`` the
+    list is cut to that many spans (flag ST_OVERFLOW) and padded with (0, 0).
+    Returns (spans int32 [k, 2], status bits)."""
+    lines = np.asarray(lines, dtype=np.int64).reshape(-1, 2)
+    out = [(0, int(prefix_len)), (int(line_start), int(ctx_len))]
+    status = 0
+    for lo, hi in np.asarray(refs, dtype=np.int64).reshape(-1, 2):
+        lo, hi = int(lo), int(hi)
+        if lo == hi and lo < 0:
+            k = len(lines) + lo
+            if k < 0:
+                status |= ST_BAD_REF
+            else:
+                out.append(tuple(int(x) for x in lines[k]))
+        elif 0 <= lo <= hi:
+            for a in range(lo, hi + 1):
+                if a >= len(anchor_line) or not (0 <= int(anchor_line[a]) < len(lines)):
+                    status |= ST_BAD_REF
+                else:
+                    out.append(tuple(int(x) for x in lines[int(anchor_line[a])]))
+        else:
+            status |= ST_BAD_REF
+    if span_stride is not None:
+        if len(out) > span_stride:
+            status |= ST_OVERFLOW
+            out = out[:span_stride]
+        out = out + [(0, 0)] * (span_stride - len(out))
+    return np.asarray(out, dtype=np.int32).reshape(-1, 2), status
 
 
 def spans_to_blockmask(spans, n: int, bs: int):
