@@ -56,8 +56,10 @@ enum {
   SSA_DEV_BAD_INDEX = 8,   /* an index entry was outside [0, ctx_len): skipped     */
   SSA_DEV_BAD_COUNT = 16,  /* counts[b] > max_selected or ctx_lens[b] > max_ctx:
                               clamped                                              */
-  SSA_DEV_TOO_MANY_SPANS = 32 /* a request had more than SSA_MAX_SPANS_PER_SEQ
+  SSA_DEV_TOO_MANY_SPANS = 32, /* a request had more than SSA_MAX_SPANS_PER_SEQ
                               spans; the surplus was ignored                       */
+  SSA_DEV_BAD_REF = 64     /* a reference named an anchor or line that does not
+                              exist, or was malformed: skipped                     */
 };
 
 #define SSA_MAX_SPANS_PER_SEQ 2048
@@ -178,6 +180,46 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q,
                               const int32_t* ctx_lens, void* out, float* lse,
                               void* workspace, size_t workspace_bytes,
                               uint32_t* dev_status, void* stream);
+
+/*
+ * Anchors and references -> span lists: the step before ssa_spans_to_index
+ * (Sec. "Self-selected attention span": anchors identify groups of contiguous
+ * tokens, the model names the anchors it needs, generation attends to the
+ * named groups; the worked arithmetic and summarization examples: "[-1]" is
+ * the previous line, the instruction is always attended, the line being
+ * generated attends to itself).  The paper gives no algorithm; the rules are:
+ * request b attends to
+ *   - its prefix           [0, prefix_len[b])                 (instruction)
+ *   - its current line     [line_start[b], ctx_lens[b])
+ *   - for every reference (lo, hi) in refs[ref_offsets[b] .. ref_offsets[b+1]):
+ *       0 <= lo <= hi      the lines identified by anchors lo..hi: line
+ *                          anchor_line[anchor_offsets[b] + a] of the request
+ *       lo == hi == -k     the k-th completed line before the current one
+ *     where the request's completed lines are the (start, end) pairs
+ *     lines[line_offsets[b] .. line_offsets[b+1]) in order of appearance.
+ * Output, ready for ssa_spans_to_index: span_offsets_out[b] = b*span_stride
+ * (B+1 entries) and, in row b of spans_out, the spans in the order above,
+ * padded with (0, 0) to span_stride pairs.  References to anchors or lines
+ * that do not exist and pairs of any other form are skipped
+ * (SSA_DEV_BAD_REF); more than span_stride spans keep the first
+ * (SSA_DEV_OVERFLOW).  All pointers dev int32; pair arrays 8-byte aligned.
+ * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE (B <= 0, span_stride < 2),
+ * SSA_ERR_ALIGN, SSA_ERR_CUDA.
+ */
+typedef struct {
+  const int32_t* line_offsets;    /* [B+1] */
+  const int32_t* lines;           /* (start, end) pairs */
+  const int32_t* anchor_offsets;  /* [B+1] */
+  const int32_t* anchor_line;     /* anchor id -> index of its line within the request */
+  const int32_t* ref_offsets;     /* [B+1] */
+  const int32_t* refs;            /* (lo, hi) pairs */
+  const int32_t* prefix_len;      /* [B] */
+  const int32_t* line_start;      /* [B] */
+  const int32_t* ctx_lens;        /* [B] */
+} ssa_anchor_tables;
+
+int32_t ssa_refs_to_spans(const ssa_anchor_tables* tables, int32_t B, int32_t* span_offsets_out,
+                          int32_t* spans_out, int32_t span_stride, uint32_t* dev_status, void* stream);
 
 /*
  * The paper's own metadata format (Sec. "CUDA Kernel Design", Attention span

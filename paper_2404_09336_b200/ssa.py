@@ -18,6 +18,7 @@ from . import build as _build
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA, ERR_UNSUPPORTED = range(1, 9)
 DEV_BAD_SPAN, DEV_CLIPPED, DEV_OVERFLOW, DEV_BAD_INDEX, DEV_BAD_COUNT, DEV_TOO_MANY_SPANS = 1, 2, 4, 8, 16, 32
+DEV_BAD_REF = 64
 MAX_SPANS_PER_SEQ = 2048
 F16, BF16, F32 = 0, 1, 2
 _DTYPES = {torch.float16: F16, torch.bfloat16: BF16, torch.float32: F32}
@@ -47,6 +48,12 @@ class Step(C.Structure):
     ]
 
 
+class AnchorTables(C.Structure):
+    """ssa_anchor_tables (see include/ssa.h)."""
+    _fields_ = [(n, C.c_void_p) for n in ("line_offsets", "lines", "anchor_offsets", "anchor_line", "ref_offsets",
+                                          "refs", "prefix_len", "line_start", "ctx_lens")]
+
+
 class SsaError(RuntimeError):
     def __init__(self, fn, code):
         self.code = code
@@ -73,6 +80,8 @@ def _load():
     lib.ssa_decode_attn_blockmask.restype = C.c_int32
     lib.ssa_decode_attn_blockmask.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
                                               C.c_int32, vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_refs_to_spans.restype = C.c_int32
+    lib.ssa_refs_to_spans.argtypes = [C.POINTER(AnchorTables), C.c_int32, vp, vp, C.c_int32, vp, vp]
     lib.ssa_decode_step.restype = C.c_int32
     lib.ssa_decode_step.argtypes = [C.POINTER(AttnDesc), C.POINTER(Step), vp]
     lib.ssa_decode_attn_sparse_noalloc.restype = C.c_int32
@@ -196,6 +205,19 @@ def decode_attn_blockmask(desc, q, k_cache, v_cache, ctx_lens, block_idx, block_
                                        int(block_size), int(max_blocks), _ptr(out), _ptr(lse), _ptr(workspace),
                                        ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_blockmask", rc, check)
+
+
+def refs_to_spans(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
+                  ctx_lens, span_offsets_out, spans_out, dev_status=None, stream=None, check=True):
+    """ssa_refs_to_spans: spans_out[B, span_stride, 2] and span_offsets_out[B+1] are written."""
+    t = AnchorTables()
+    for name, ten in (("line_offsets", line_offsets), ("lines", lines), ("anchor_offsets", anchor_offsets),
+                      ("anchor_line", anchor_line), ("ref_offsets", ref_offsets), ("refs", refs),
+                      ("prefix_len", prefix_len), ("line_start", line_start), ("ctx_lens", ctx_lens)):
+        setattr(t, name, None if ten is None else ten.data_ptr())
+    rc = lib.ssa_refs_to_spans(C.byref(t), int(ctx_lens.numel()), _ptr(span_offsets_out), _ptr(spans_out),
+                               int(spans_out.shape[1]), _ptr(dev_status), _stream(stream))
+    return _check("ssa_refs_to_spans", rc, check)
 
 
 def make_step(span_offsets, spans, ctx_lens, index, counts, q, k_cache, v_cache, max_selected, out, lse=None,

@@ -1,0 +1,126 @@
+"""ssa_refs_to_spans against the oracle (bit-exact span rows), and the whole
+chain references -> spans -> index lists -> attention on the device."""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssa_oracle as O
+from paper_2404_09336_b200 import ssa
+
+from gpu_util import DEV, Problem
+from parity import assert_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def flat(lists, width):
+    offs = np.zeros(len(lists) + 1, np.int32)
+    offs[1:] = np.cumsum([len(x) for x in lists])
+    data = np.asarray([v for x in lists for v in x], np.int32).reshape(-1, width) if offs[-1] else \
+        np.zeros((1, width), np.int32)
+    return torch.from_numpy(offs).to(DEV), torch.from_numpy(np.ascontiguousarray(data)).to(DEV)
+
+
+def run_refs(reqs, stride):
+    """reqs: list of dicts(lines, anchors, refs, prefix, start, ctx)."""
+    B = len(reqs)
+    lo, ld = flat([r["lines"] for r in reqs], 2)
+    ao, ad = flat([[(a,) for a in r["anchors"]] for r in reqs], 1)
+    ro, rd = flat([r["refs"] for r in reqs], 2)
+    i32 = lambda k: torch.tensor([r[k] for r in reqs], dtype=torch.int32, device=DEV)
+    prefix, start, ctx = i32("prefix"), i32("start"), i32("ctx")
+    so = torch.full((B + 1,), -7, dtype=torch.int32, device=DEV)
+    sp = torch.full((B, stride, 2), -7, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ssa.refs_to_spans(lo, ld, ao, ad.view(-1), ro, rd, prefix, start, ctx, so, sp, status)
+    torch.cuda.synchronize()
+    return so, sp, ctx, int(status.item())
+
+
+def compare(reqs, stride):
+    so, sp, ctx, status = run_refs(reqs, stride)
+    want_status = 0
+    for b, r in enumerate(reqs):
+        ref, st = O.resolve_references(r["lines"], r["anchors"], r["refs"], r["prefix"], r["start"], r["ctx"], stride)
+        want_status |= st
+        assert sp[b].cpu().numpy().tolist() == ref.tolist(), f"request {b}"
+    assert so.cpu().numpy().tolist() == [b * stride for b in range(len(reqs) + 1)]
+    gpu_bits = {O.ST_OVERFLOW: ssa.DEV_OVERFLOW, O.ST_BAD_REF: ssa.DEV_BAD_REF}
+    assert status == sum(v for k, v in gpu_bits.items() if want_status & k)
+    return so, sp, ctx
+
+
+def test_paper_examples_and_flags():
+    arith = dict(lines=[(0, 14), (14, 40), (40, 54), (54, 66)], anchors=[0, 2, 3], refs=[(0, 0), (1, 1), (2, 2)],
+                 prefix=0, start=66, ctx=69)
+    summ = dict(lines=[(12 + 8 * i, 20 + 8 * i) for i in range(31)] + [(260, 280)], anchors=list(range(31)),
+                refs=[(17, 19), (-1, -1)], prefix=12, start=280, ctx=291)
+    so, sp, ctx = compare([arith, summ], 8)
+    # union of the resolved spans = the positions the paper's examples attend to
+    assert O.spans_to_index(sp[0].cpu().numpy(), 69).tolist() == list(range(0, 14)) + list(range(40, 69))
+    assert O.spans_to_index(sp[1].cpu().numpy(), 291).tolist() == \
+        list(range(0, 12)) + list(range(148, 172)) + list(range(260, 291))
+    compare([dict(arith, refs=[(0, 2), (-1, -1), (-2, -2), (-4, -4)])], 5)          # overflow: 2 + 6 spans
+    for bad in ([(5, 5)], [(-9, -9)], [(1, 0)], [(-1, 2)], [(0, 7)]):
+        compare([dict(arith, refs=bad)], 8)
+    compare([dict(lines=[], anchors=[], refs=[], prefix=3, start=3, ctx=9)], 2)
+    compare([dict(arith, anchors=[0, 9, 3])], 8)                                    # an anchor that points nowhere
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_fuzz(seed):
+    rnd = random.Random(seed)
+    reqs = []
+    for _ in range(rnd.randint(1, 30)):
+        n_lines = rnd.randint(0, 50)
+        pos, lines = rnd.randint(0, 20), []
+        prefix = pos
+        for _ in range(n_lines):
+            ln = rnd.randint(1, 30)
+            lines.append((pos, pos + ln))
+            pos += ln + rnd.randint(0, 2)
+        anchors = [rnd.randint(-1, n_lines) for _ in range(rnd.randint(0, 20))]
+        refs = []
+        for _ in range(rnd.randint(0, 40)):
+            if rnd.random() < 0.3:
+                k = -rnd.randint(1, n_lines + 2)
+                refs.append((k, k))
+            else:
+                a = rnd.randint(-1, len(anchors) + 1)
+                refs.append((a, a + rnd.randint(-1, 4)))
+        reqs.append(dict(lines=lines, anchors=anchors, refs=refs, prefix=prefix, start=pos, ctx=pos + rnd.randint(0, 9)))
+    compare(reqs, rnd.choice([4, 32, 100]))
+
+
+def test_references_to_attention_on_the_device():
+    rnd = random.Random(3)
+    B, H, T, D = 4, 2, 900, 128
+    p = Problem(B, H, T, D, "bf16", seed=5)
+    reqs = []
+    for b in range(B):
+        lines = [(20 + 40 * i, 60 + 40 * i) for i in range(18)]
+        refs = [(rnd.randint(0, 8), rnd.randint(9, 17)), (-1, -1)] if b else [(3, 3)]
+        reqs.append(dict(lines=lines, anchors=list(range(18)), refs=refs, prefix=20, start=740, ctx=760 + 30 * b))
+    stride = 32
+    so, sp, ctx, status = run_refs(reqs, stride)
+    assert status == 0
+    index = torch.full((B, T), -7, dtype=torch.int32, device=DEV)
+    counts = torch.zeros(B, dtype=torch.int32, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ssa.spans_to_index(so, sp.view(-1, 2), ctx, index, counts, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ctx_l = [r["ctx"] for r in reqs]
+    out, lse, status, _ = p.sparse(ctx_l, index.cpu().numpy(), counts.cpu().numpy().tolist(), max_selected=T)
+    want_idx = np.full((B, T), -1, np.int32)
+    want_cnt = []
+    for b, r in enumerate(reqs):
+        spans, _ = O.resolve_references(r["lines"], r["anchors"], r["refs"], r["prefix"], r["start"], r["ctx"])
+        idx = O.spans_to_index(spans, r["ctx"])
+        want_idx[b, :len(idx)] = idx
+        want_cnt.append(len(idx))
+    assert counts.cpu().numpy().tolist() == want_cnt
+    ref, _ = O.decode_attn_sparse(p.q_bits, p.k_bits, p.v_bits, ctx_l, want_idx, want_cnt, 1 / np.sqrt(D), "bf16")
+    assert_parity(out, ref, False, "references to attention")
