@@ -262,6 +262,32 @@ def test_strided_views_and_launch_counter():
     assert_parity(out, ref, False, "strided q")
 
 
+def test_mixed_batch_of_full_context_and_restricted_requests():
+    # requests at a "determine span" step attend to everything, the others to their spans, in one launch
+    wl = inputs.make_config(2, B=6, H=4)
+    spans, offs = [], [0]
+    for i in range(wl.B):
+        sp = [(0, int(wl.ctx_lens[i]))] if i % 2 == 0 else wl.spans_of(i).tolist()
+        spans += sp
+        offs.append(len(spans))
+    wl.spans, wl.span_offsets = np.asarray(spans, np.int32), np.asarray(offs, np.int32)
+    ds = DecodeStep(wl, out_dtype=torch.float32)
+    assert ds.max_selected == int(wl.ctx_lens[::2].max())
+    ds.step()
+    torch.cuda.synchronize()
+    got = ds.out_f64()
+    k, v = wl.kv_bits()
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, ds.index_stride)
+    ref, _ = O.decode_attn_sparse(wl.q_bits(), k, v, wl.ctx_lens, index, counts, scale_of(wl.D), wl.dtype)
+    refd, _ = O.decode_attn_dense(wl.q_bits(), k, v, wl.ctx_lens, scale_of(wl.D), wl.dtype)
+    assert int(ds.status.item()) == 0
+    assert_parity(got, ref, False, "mixed batch")
+    assert_parity(got[::2], refd[::2], False, "full-context requests")
+    ds.attend_dense()
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(ds.out_f64()[::2], got[::2], rtol=0, atol=1e-5)
+
+
 def test_decode_step_in_one_call_with_host_copies():
     # ssa_decode_step: copy in, index, attention, copy out - against the two separate calls
     wl = inputs.make_config(2, B=5, H=4)
