@@ -40,7 +40,7 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kU = SSA_U;              // 32-byte loads in flight per lane, per tensor
 constexpr int kMaxChunk = 512;         // index entries staged per block
 constexpr int kIdxPerThread = kMaxChunk / kThreads;
-constexpr int kMaskChunk = 256;        // positions a block expands from bitmasks
+constexpr int kMaskChunk = 512;        // positions a block expands from bitmasks
 enum { kDense = 0, kIndex = 1, kBlockMask = 2 };
 
 struct DecodeParams {
