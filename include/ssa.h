@@ -78,7 +78,9 @@ typedef enum { SSA_F16 = 0, SSA_BF16 = 1, SSA_F32 = 2 } ssa_dtype;
  * caller before the call; it is attended only if selected.
  * Supported: D in {64, 128}; kv_dtype F16 or BF16 (q has the same type);
  * out_dtype equal to kv_dtype or F32; H_kv == H (multi-head attention, as in
- * the paper's LLaMA-7B).  Every base pointer and every stride * element size
+ * the paper's LLaMA-7B) or H_kv dividing H (grouped queries, not in the paper:
+ * query head h reads K/V head h / (H/H_kv); the cache then has H_kv heads).
+ * Every base pointer and every stride * element size
  * must be a multiple of 16 bytes.
  */
 typedef struct {

@@ -61,6 +61,7 @@ struct DecodeParams {
   int64_t q_sb, q_sh, k_sb, k_sh, v_sb, v_sh, o_sb, o_sh;
   uint32_t k_row_bytes, v_row_bytes;   // token stride of the cache in bytes
   int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32, early_release;
+  int32_t kv_group;         // query heads per K/V head (1: multi-head attention)
   float scale_log2;         // softmax scale * log2(e)
 };
 
@@ -214,9 +215,9 @@ decode_partial_kernel(const DecodeParams p) {
   }
 
   const char* kbase = reinterpret_cast<const char*>(
-      reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)h * p.k_sh + col * 16);
+      reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)(h / p.kv_group) * p.k_sh + col * 16);
   const char* vbase = reinterpret_cast<const char*>(
-      reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)h * p.v_sh + col * 16);
+      reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)(h / p.kv_group) * p.v_sh + col * 16);
 
   float2 q2[8];
 #pragma unroll
@@ -389,7 +390,7 @@ static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 1
 static int32_t check_desc(const ssa_attn_desc* d) {
   if (d->B <= 0 || d->H <= 0 || d->max_ctx <= 0 || d->B > 65535 || d->H > 65535) return SSA_ERR_SHAPE;
   if (d->D != 64 && d->D != 128) return SSA_ERR_UNSUPPORTED;
-  if (d->H_kv != d->H) return SSA_ERR_UNSUPPORTED;
+  if (d->H_kv <= 0 || d->H % d->H_kv != 0) return SSA_ERR_UNSUPPORTED;
   if (d->kv_dtype != SSA_F16 && d->kv_dtype != SSA_BF16) return SSA_ERR_DTYPE;
   if (d->out_dtype != d->kv_dtype && d->out_dtype != SSA_F32) return SSA_ERR_DTYPE;
   const int64_t strides[] = {d->q_stride_b, d->q_stride_h, d->k_stride_b, d->k_stride_t, d->k_stride_h,
@@ -475,6 +476,7 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   p.ws_ml = reinterpret_cast<float2*>(reinterpret_cast<char*>(ws) + pl.acc_bytes);
   p.dev_status = dev_status;
   p.q_sb = d->q_stride_b; p.q_sh = d->q_stride_h;
+  p.kv_group = d->H / d->H_kv;
   p.k_sb = d->k_stride_b; p.k_sh = d->k_stride_h;
   p.v_sb = d->v_stride_b; p.v_sh = d->v_stride_h;
   p.k_row_bytes = (uint32_t)(d->k_stride_t * 2);

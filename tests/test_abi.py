@@ -82,7 +82,7 @@ def test_sparse_rejects_bad_arguments_without_launching():
     assert sparse(d, k=C.c_void_p(0x1008)) == ssa.ERR_ALIGN
     assert sparse(d, ws=NUL) == ssa.ERR_WORKSPACE
     assert sparse(d, ws_bytes=16) == ssa.ERR_WORKSPACE
-    for field, val, err in [("D", 96, ssa.ERR_UNSUPPORTED), ("H_kv", 2, ssa.ERR_UNSUPPORTED),
+    for field, val, err in [("D", 96, ssa.ERR_UNSUPPORTED), ("H_kv", 3, ssa.ERR_UNSUPPORTED),
                             ("kv_dtype", ssa.F32, ssa.ERR_DTYPE), ("out_dtype", ssa.F16, ssa.ERR_DTYPE),
                             ("k_stride_t", 132, ssa.ERR_ALIGN), ("B", 0, ssa.ERR_SHAPE),
                             ("max_ctx", 0, ssa.ERR_SHAPE), ("v_stride_h", -128, ssa.ERR_SHAPE)]:

@@ -262,6 +262,31 @@ def test_strided_views_and_launch_counter():
     assert_parity(out, ref, False, "strided q")
 
 
+def test_grouped_query_heads_share_a_kv_head():
+    # not in the paper (LLaMA-7B is multi-head): H = 8 query heads over H_kv = 2 cache heads
+    B, H, Hkv, T, D = 3, 8, 2, 700, 128
+    p = Problem(B, Hkv, T, D, "bf16", seed=31)               # cache with H_kv heads
+    rng = np.random.default_rng(2)
+    from gpu_util import random_bits
+    p.q_bits = random_bits(rng, (B, H, D), "bf16")
+    p.H = H
+    p.upload()
+    ctx = [700, 333, 64]
+    counts = [300, 120, 64]
+    index = np.full((B, 704), -1, np.int32)
+    for b in range(B):
+        index[b, :counts[b]] = np.sort(rng.choice(ctx[b], counts[b], replace=False))
+    out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=700)
+    k_rep, v_rep = np.repeat(p.k_bits, H // Hkv, axis=1), np.repeat(p.v_bits, H // Hkv, axis=1)
+    ref, ref_lse = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, index, counts, scale_of(D), "bf16")
+    assert status == 0
+    assert_parity(out, ref, False, "grouped queries")
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+    out_d, _, _ = p.dense(ctx)
+    ref_d, _ = O.decode_attn_dense(p.q_bits, k_rep, v_rep, ctx, scale_of(D), "bf16")
+    assert_parity(out_d, ref_d, False, "grouped queries, dense")
+
+
 def test_mixed_batch_of_full_context_and_restricted_requests():
     # requests at a "determine span" step attend to everything, the others to their spans, in one launch
     wl = inputs.make_config(2, B=6, H=4)
