@@ -341,3 +341,48 @@ def test_decode_step_in_one_call_with_host_copies():
     st = ssa.make_step(ds.span_offsets, ds.spans, ds.ctx_lens, ds.index, ds.counts, ds.q, ds.k, ds.v,
                        ds.max_selected, ds.out, ds.lse, None, ds.status)
     assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_WORKSPACE
+
+
+def test_side_stream_graph_replay_and_determinism():
+    wl = inputs.make_config(3, B=2, H=4)
+    ds = DecodeStep(wl, out_dtype=torch.float32)
+    ds.step()
+    torch.cuda.synchronize()
+    first = ds.out.clone()
+    # twice the same call: bit-identical (no atomics in the accumulation)
+    ds.out.zero_()
+    ds.step()
+    torch.cuda.synchronize()
+    assert torch.equal(ds.out, first)
+    # on a side stream, handed over explicitly and as torch's current stream
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    ds.out.zero_()
+    torch.cuda.synchronize()
+    ds.step(stream=side)
+    side.synchronize()
+    assert torch.equal(ds.out, first)
+    ds.out.zero_()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        ds.step()
+    side.synchronize()
+    assert torch.equal(ds.out, first)
+    # captured into a CUDA graph and replayed
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        ds.step()
+    ds.out.zero_()
+    ds.counts.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(ds.out, first) and int(ds.status.item()) == 0
+    # the no-workspace and the dense calls through the same graph mechanism
+    g2 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g2, stream=side):
+        ds.attend_dense()
+    g2.replay()
+    torch.cuda.synchronize()
+    k, v = wl.kv_bits()
+    refd, _ = O.decode_attn_dense(wl.q_bits(), k, v, wl.ctx_lens, scale_of(wl.D), wl.dtype)
+    assert_parity(ds.out_f64(), refd, False, "dense from a graph")

@@ -164,3 +164,26 @@ def test_end_to_end_on_device_and_bad_bits():
     hc[2] = stride + 5
     _, _, st3 = attention_from_lists(p, wl.ctx_lens.tolist(), hb, hm, hc, bs, stride)
     assert st3 & ssa.DEV_BAD_COUNT
+
+
+def test_full_size_workload_through_the_blocked_lists():
+    # cfg 3 at full size in the launch configuration of the benchmark; sampled outputs against the oracle
+    from paper_2404_09336_b200.runner import DecodeStep
+    wl = inputs.make_config(3)
+    ds = DecodeStep(wl)
+    ds.enable_blockmask(256)
+    ds.step_blockmask()
+    torch.cuda.synchronize()
+    assert int(ds.status.item()) == 0
+    got = ds.out_f64()
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, 4096)
+    q = wl.q_bits()
+    for b in (3, 12):
+        k, v = wl.kv_bits_seq(b)
+        ref, _ = O.decode_attn_sparse(q[b:b + 1], k[None], v[None], wl.ctx_lens[b:b + 1], index[b:b + 1],
+                                      counts[b:b + 1], 1 / np.sqrt(wl.D), wl.dtype, heads=[0, 17, 31])
+        for h in (0, 17, 31):
+            assert_parity(got[b, h], ref[0, h], True, f"request {b} head {h}")
+    ds.step()
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(ds.out_f64(), got, rtol=0, atol=4e-3)       # bf16 outputs of the two paths
