@@ -124,3 +124,54 @@ def test_references_to_attention_on_the_device():
     assert counts.cpu().numpy().tolist() == want_cnt
     ref, _ = O.decode_attn_sparse(p.q_bits, p.k_bits, p.v_bits, ctx_l, want_idx, want_cnt, 1 / np.sqrt(D), "bf16")
     assert_parity(out, ref, False, "references to attention")
+
+
+def test_generation_loop_with_growing_context():
+    # several consecutive decode steps as a generation loop makes them: the context grows by one row per
+    # step, the current line grows with it, every third step is a "determine span" step over everything
+    B, H, T, D = 3, 2, 400, 128
+    p = Problem(B, H, T, D, "bf16", seed=8)
+    lines = [(16 + 30 * i, 46 + 30 * i) for i in range(8)]                     # completed lines, 16..256
+    reqs = [dict(lines=lines, anchors=list(range(8)), refs=[(b, b + 2), (-1, -1)], prefix=16, start=256,
+                 ctx=300 + 7 * b) for b in range(B)]
+    lo, ld = flat([r["lines"] for r in reqs], 2)
+    ao, ad = flat([[(a,) for a in r["anchors"]] for r in reqs], 1)
+    ro, rd = flat([r["refs"] for r in reqs], 2)
+    full_ro = torch.zeros(B + 1, dtype=torch.int32, device=DEV)                # no references: prefix + line only
+    i32 = lambda vals: torch.tensor(vals, dtype=torch.int32, device=DEV)
+    prefix, start = i32([r["prefix"] for r in reqs]), i32([r["start"] for r in reqs])
+    zero = i32([0] * B)
+    ctx = i32([r["ctx"] for r in reqs])
+    stride = 16
+    so = torch.zeros(B + 1, dtype=torch.int32, device=DEV)
+    sp = torch.zeros((B, stride, 2), dtype=torch.int32, device=DEV)
+    index = torch.zeros((B, T), dtype=torch.int32, device=DEV)
+    counts = torch.zeros(B, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = torch.zeros((B, H, D), dtype=torch.float32, device=DEV)
+    desc = ssa.make_desc(p.q, p.k, p.v, out)
+    ws = torch.empty(ssa.decode_workspace_bytes(desc, T), dtype=torch.uint8, device=DEV)
+    for step in range(7):
+        determine = step % 3 == 0
+        if determine:       # the whole context: an empty prefix and a "line" that starts at 0
+            ssa.refs_to_spans(lo, ld, ao, ad.view(-1), full_ro, rd, zero, zero, ctx, so, sp, status)
+        else:
+            ssa.refs_to_spans(lo, ld, ao, ad.view(-1), ro, rd, prefix, start, ctx, so, sp, status)
+        ssa.spans_to_index(so, sp.view(-1, 2), ctx, index, counts, status)
+        ssa.decode_attn_sparse(desc, p.q, p.k, p.v, ctx, index, counts, T, out, None, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ctx_l = ctx.cpu().tolist()
+        want_idx, want_cnt = np.full((B, T), -1, np.int32), []
+        for b, r in enumerate(reqs):
+            if determine:
+                idx = np.arange(ctx_l[b], dtype=np.int32)
+            else:
+                spans, _ = O.resolve_references(r["lines"], r["anchors"], r["refs"], r["prefix"], r["start"], ctx_l[b])
+                idx = O.spans_to_index(spans, ctx_l[b])
+            want_idx[b, :len(idx)] = idx
+            want_cnt.append(len(idx))
+        assert counts.cpu().tolist() == want_cnt
+        ref, _ = O.decode_attn_sparse(p.q_bits, p.k_bits, p.v_bits, ctx_l, want_idx, want_cnt, 1 / np.sqrt(D), "bf16")
+        assert_parity(out.double().cpu().numpy(), ref, False, f"step {step}")
+        ctx += 1                                                               # the next token's row is appended
