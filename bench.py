@@ -72,7 +72,7 @@ def hbm_peak():
 # clocks
 # ---------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("clocks.mem,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -99,7 +99,7 @@ class ClockSampler:
                 self.proc.wait(timeout=5)
             except Exception:
                 self.proc.kill()
-        sm, mx, reasons, n_all = [], 0.0, set(), 0
+        sm, mem, mx, reasons, n_all = [], [], 0.0, set(), 0
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for t, line in self.rows:
             parts = [p.strip() for p in line.split(",")]
@@ -110,6 +110,7 @@ class ClockSampler:
                 continue
             try:
                 sm.append(float(parts[1]))
+                mem.append(float(parts[0]))
                 mx = max(mx, float(parts[2]))
             except ValueError:
                 continue
@@ -117,6 +118,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx or None,
+                "mem_mhz": statistics.median(mem) if mem else None,
                 "reasons": sorted(reasons), "samples_under_load": len(sm), "samples": n_all}
 
 
@@ -281,6 +283,10 @@ def measure(torch, ssa, timer, ds, steps, warmup, peak, kernel_pass=True):
     # (a) direct calls through the binding
     ms = timer.run(lambda i: (rot(i), ds.step()), steps)
     res["direct_us"] = ms / steps * 1e3
+    # the same without rotating: every step re-reads copy 0 (L2-warm where the selection fits the L2)
+    ds.select_copy(0)
+    ms = timer.run(lambda i: ds.step(), steps)
+    res["warm_us"] = ms / steps * 1e3
     # (b) the same step replayed from CUDA graphs (one per KV copy)
     graphs = capture_graphs(torch, ds, ds.step)
     for g in graphs:
@@ -466,7 +472,8 @@ def run_ours(args):
         "pct_hbm_peak_measured": 100 * value / world / peak, "pct_hbm_peak_spec": 100 * value / world / SPEC_HBM_GBS,
         "speedup_vs_dense": main["speedup_vs_dense"], "density": main["density"],
         "us_per_step": ms / steps * 1e3,
-        "breakdown_us": {k: main[k] for k in ("direct_us", "graph_us", "index_us", "sparse_attn_us", "dense_us")},
+        "breakdown_us": {k: main[k] for k in ("direct_us", "graph_us", "index_us", "sparse_attn_us", "dense_us",
+                                              "warm_us")},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "us_per_step": ms_e2e / steps * 1e3,
@@ -506,7 +513,7 @@ def run_ours(args):
                 sweep.append(r)
                 del d
             torch.cuda.empty_cache()
-        keep = ("workload", "density", "selected_bytes", "step_us", "index_us", "sparse_attn_us", "dense_us", "gbs",
+        keep = ("workload", "density", "selected_bytes", "step_us", "warm_us", "index_us", "sparse_attn_us", "dense_us", "gbs",
                 "attn_gbs", "dense_gbs", "pct_peak_measured", "pct_peak_spec", "speedup_vs_dense", "launch_mode",
                 "kv_copies")
         line["sweep"] = [{k: (round(r[k], 4) if isinstance(r[k], float) else r[k]) for k in keep} for r in sweep]
