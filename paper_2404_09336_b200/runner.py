@@ -172,6 +172,8 @@ class DecodeStep:
         """Decode step whose per-step inputs start in pinned host memory and
         whose result ends there (ssa_decode_step with both copies); the KV
         cache is the resident state."""
+        if not hasattr(self, "h_in"):
+            raise RuntimeError("call make_host_buffers() before step_from_host()")
         key = (self.k.data_ptr(), self.max_selected)
         st = self._host_steps.get(key)
         if st is None:
