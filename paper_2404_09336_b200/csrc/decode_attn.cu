@@ -360,9 +360,13 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   if (!d || d->B <= 0 || d->H <= 0 || max_selected <= 0) return false;
   if (d->D != 64 && d->D != 128) return false;
   const long long units = (long long)d->B * d->H;
-  const long long want = 148 * 8;                     // blocks for one full wave
+  // The second pass costs about as much as two rounds of a block, so a request is split only when that buys
+  // parallelism: one chunk whenever the list fits a block's staging area and either every SM gets a block or
+  // the list is short anyway; otherwise 256-entry chunks, halved while the grid has under two blocks per SM.
+  const long long want = 148 * 2;
   int chunk = 256;
-  while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
+  if (max_selected <= kMaxChunk && (units >= 148 || max_selected <= 256)) chunk = kMaxChunk;
+  else while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
   int n_chunks = (max_selected + chunk - 1) / chunk;
   if (n_chunks == 1) chunk = (max_selected + 31) / 32 * 32;
   pl->chunk = chunk;

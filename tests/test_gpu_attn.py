@@ -147,6 +147,31 @@ def test_multi_chunk_merge_and_tail_sizes():
             np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
 
 
+@pytest.mark.parametrize("B,H", [(2, 2), (5, 32)])
+def test_one_chunk_or_several_on_both_sides_of_the_switch(B, H):
+    # the host picks one chunk per request or several from (B*H, max_selected): list lengths and contexts
+    # right below and above the sizes where that choice changes, for few and for many (request, head) pairs
+    D = 128
+    rng = np.random.default_rng(B)
+    for T in (256, 257, 512, 513):
+        p = Problem(B, H, T, D, "bf16", seed=T + B)
+        ctx = [T] * B
+        counts = [T] + [int(rng.integers(1, T + 1)) for _ in range(B - 1)]
+        index = np.full((B, T + 7), -1, np.int32)
+        for b in range(B):
+            index[b, :counts[b]] = np.sort(rng.choice(T, counts[b], replace=False))
+        out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=T)
+        ref, ref_lse = oracle_sparse(p, ctx, index, counts)
+        assert status == 0
+        assert_parity(out, ref, False, f"sparse T={T}")
+        np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+        out_d, lse_d, st_d = p.dense(ctx)
+        ref_d, ref_lse_d = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, ctx, scale_of(D), "bf16")
+        assert st_d == 0
+        assert_parity(out_d, ref_d, False, f"dense T={T}")
+        np.testing.assert_allclose(lse_d, ref_lse_d, rtol=1e-5, atol=1e-5)
+
+
 def test_large_batch_of_short_ragged_requests():
     # thousands of requests, one head each, lengths 0..600: several chunks per request, many empty ones
     B, H, T, D = 4100, 1, 600, 64
