@@ -156,6 +156,9 @@ size_t ssa_decode_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selecte
  *   ctx_lens   dev int32 [B]
  *   index      dev int32 [B * index_stride];  counts dev int32 [B]
  *   out        dev, out_dtype (written);  lse dev float [B*H] or NULL (written)
+ *              (both are only ever stored to, once per element, so they may
+ *              also be page-locked host memory that the device addresses: a
+ *              row then crosses the bus as soon as it is finished)
  *   workspace  dev, >= ssa_decode_workspace_bytes(desc, max_selected) bytes,
  *              16-byte aligned
  * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE, SSA_ERR_DTYPE, SSA_ERR_ALIGN,
@@ -283,9 +286,26 @@ int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, cons
  * to host_out after the attention kernels.  Host arenas should be page-locked,
  * otherwise the copies are not asynchronous.  The call does not wait for any of
  * this work.  The KV cache is resident state and is never copied.
+ *
+ * flags = 0: both copies are cudaMemcpyAsync transfers (copy engine).
+ * flags = SSA_STEP_COPY_BY_KERNEL: both copies are done by a kernel of the
+ * library that reads / writes the host arena across the bus.  For the few
+ * hundred KB that change per decode step this is faster than a copy-engine
+ * transfer, whose set-up time dominates at that size.  The host arenas must
+ * then be page-locked memory that the device addresses under the same pointer
+ * (cudaHostAlloc / cudaMallocHost under unified addressing; checked with
+ * cudaPointerGetAttributes, else SSA_ERR_UNSUPPORTED), all four arena pointers
+ * 16-byte aligned and both sizes multiples of 16 (else SSA_ERR_ALIGN); these
+ * checks come first, so a refused call has enqueued nothing.
+ * In either mode `out` and `lse` may themselves point into such host memory:
+ * the attention kernels then store each finished row straight across the bus
+ * while the rest of the batch is still being read, and the copy out only has
+ * to carry what kernels also read back (counts, the status word).
  * Errors: SSA_ERR_NULL for a NULL desc/step or an inconsistent copy request,
- * otherwise those of the two calls; nothing after a failing stage is enqueued.
+ * SSA_ERR_UNSUPPORTED for unknown flag bits, otherwise those of the two calls;
+ * nothing after a failing stage is enqueued.
  */
+#define SSA_STEP_COPY_BY_KERNEL 1u
 typedef struct {
   const int32_t* span_offsets;  /* dev [B+1]                                   */
   const int32_t* spans;         /* dev (start, end) pairs                      */
@@ -295,8 +315,8 @@ typedef struct {
   const void* q;                /* dev                                         */
   const void* k_cache;          /* dev                                         */
   const void* v_cache;          /* dev                                         */
-  void* out;                    /* dev                     (written)           */
-  float* lse;                   /* dev [B*H] or NULL       (written)           */
+  void* out;                    /* dev, or host the device addresses (written) */
+  float* lse;                   /* same, [B*H], or NULL    (written)           */
   void* workspace;              /* dev                                         */
   size_t workspace_bytes;
   uint32_t* dev_status;         /* dev [1] or NULL                             */
@@ -308,6 +328,7 @@ typedef struct {
   void* host_out;               /* host (pinned) or NULL                       */
   const void* dev_out;          /* dev                                         */
   size_t out_bytes;
+  uint32_t flags;               /* 0 or SSA_STEP_COPY_BY_KERNEL                */
 } ssa_step;
 
 int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* step, void* stream);

@@ -1,24 +1,84 @@
 // ssa_decode_step: one decode step (optional copy in, span lists -> index
 // lists -> span-restricted attention, optional copy out) enqueued by one call.
+#include <algorithm>
+
 #include "ssa_common.cuh"
+
+namespace ssa {
+
+// Copy of n16 16-byte words between the device and page-locked host memory the
+// device can address.  Every word is requested at once, so the transfer costs
+// about one trip over the bus plus its bytes; a copy-engine transfer of the
+// same few hundred KB pays several microseconds of set-up on top.
+__global__ void __launch_bounds__(256) copy_words_kernel(uint4* __restrict__ dst, const uint4* __restrict__ src,
+                                                          size_t n16) {
+  grid_dependency_wait();                      // the destination may still be read by the previous kernel
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride) dst[i] = src[i];
+}
+
+// True when `p` is page-locked host memory that kernels can address under the same pointer.
+static bool device_addressable_host(const void* p) {
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return a.type == cudaMemoryTypeHost && a.devicePointer == p;
+}
+
+static int32_t copy_by_kernel(void* dst, const void* src, size_t bytes, cudaStream_t st) {
+  const size_t n16 = bytes / 16;
+  const unsigned blocks = (unsigned)std::min<size_t>((n16 + 255) / 256, 148 * 4);
+  const cudaError_t err = launch_pdl(copy_words_kernel, dim3(blocks), dim3(256), st, reinterpret_cast<uint4*>(dst),
+                                     reinterpret_cast<const uint4*>(src), n16);
+  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  note_launches(1);
+  return SSA_OK;
+}
+
+static bool copy_aligned(const void* a, const void* b, size_t bytes) {
+  return bytes % 16 == 0 && reinterpret_cast<uintptr_t>(a) % 16 == 0 && reinterpret_cast<uintptr_t>(b) % 16 == 0;
+}
+
+}  // namespace ssa
 
 extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s, void* stream) {
   if (!desc || !s) return SSA_ERR_NULL;
   if (s->host_in && (!s->dev_in || s->in_bytes == 0)) return SSA_ERR_NULL;
   if (s->host_out && (!s->dev_out || s->out_bytes == 0)) return SSA_ERR_NULL;
+  if (s->flags & ~(uint32_t)SSA_STEP_COPY_BY_KERNEL) return SSA_ERR_UNSUPPORTED;
+  const bool by_kernel = (s->flags & SSA_STEP_COPY_BY_KERNEL) != 0;
+  if (by_kernel) {                             // everything is checked before anything is enqueued
+    if (s->host_in && !ssa::copy_aligned(s->host_in, s->dev_in, s->in_bytes)) return SSA_ERR_ALIGN;
+    if (s->host_out && !ssa::copy_aligned(s->host_out, s->dev_out, s->out_bytes)) return SSA_ERR_ALIGN;
+    if (s->host_in && !ssa::device_addressable_host(s->host_in)) return SSA_ERR_UNSUPPORTED;
+    if (s->host_out && !ssa::device_addressable_host(s->host_out)) return SSA_ERR_UNSUPPORTED;
+  }
   cudaStream_t st = (cudaStream_t)stream;
-  if (s->host_in &&
-      cudaMemcpyAsync(s->dev_in, s->host_in, s->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return SSA_ERR_CUDA;
-  int32_t rc = ssa_spans_to_index(s->span_offsets, s->spans, s->ctx_lens, desc->B, s->index, s->index_stride,
-                                  s->counts, s->dev_status, stream);
+  int32_t rc;
+  if (s->host_in) {
+    if (by_kernel) {
+      rc = ssa::copy_by_kernel(s->dev_in, s->host_in, s->in_bytes, st);
+      if (rc != SSA_OK) return rc;
+    } else if (cudaMemcpyAsync(s->dev_in, s->host_in, s->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+      return SSA_ERR_CUDA;
+    }
+  }
+  rc = ssa_spans_to_index(s->span_offsets, s->spans, s->ctx_lens, desc->B, s->index, s->index_stride,
+                          s->counts, s->dev_status, stream);
   if (rc != SSA_OK) return rc;
   rc = ssa_decode_attn_sparse(desc, s->q, s->k_cache, s->v_cache, s->ctx_lens, s->index, s->index_stride,
                               s->counts, s->max_selected, s->out, s->lse, s->workspace, s->workspace_bytes,
                               s->dev_status, stream);
   if (rc != SSA_OK) return rc;
-  if (s->host_out &&
-      cudaMemcpyAsync(s->host_out, s->dev_out, s->out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return SSA_ERR_CUDA;
+  if (s->host_out) {
+    if (by_kernel) {
+      rc = ssa::copy_by_kernel(const_cast<void*>(s->host_out), s->dev_out, s->out_bytes, st);
+      if (rc != SSA_OK) return rc;
+    } else if (cudaMemcpyAsync(s->host_out, s->dev_out, s->out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+      return SSA_ERR_CUDA;
+    }
+  }
   return SSA_OK;
 }

@@ -43,6 +43,6 @@ const char* ssa_status_string(int32_t status) {
   }
 }
 
-int32_t ssa_version(void) { return 100; }
+int32_t ssa_version(void) { return 101; }
 
 }  // extern "C"

@@ -26,20 +26,26 @@ def tensor_to_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
+def _nbytes(shape, dt):
+    return int(np.prod(shape)) * torch.empty((), dtype=dt).element_size()
+
+
+def _views(buf, specs):
+    """Tensors of the given (shape, dtype) laid back to back at 256-byte boundaries in the uint8 buffer."""
+    views, o = [], 0
+    for shape, dt in specs:
+        n = _nbytes(shape, dt)
+        views.append(buf[o:o + n].view(dt).view(shape))
+        o += (n + 255) // 256 * 256
+    return views
+
+
 def _arena(device, specs):
     """One uint8 device buffer holding tensors of the given (shape, dtype)
     back to back at 256-byte boundaries; returns (buffer, views)."""
-    offs, total = [], 0
-    for shape, dt in specs:
-        offs.append(total)
-        nbytes = int(np.prod(shape)) * torch.empty((), dtype=dt).element_size()
-        total += (nbytes + 255) // 256 * 256
+    total = sum((_nbytes(shape, dt) + 255) // 256 * 256 for shape, dt in specs)
     buf = torch.zeros(total, dtype=torch.uint8, device=device)
-    views = []
-    for (shape, dt), o in zip(specs, offs):
-        nbytes = int(np.prod(shape)) * torch.empty((), dtype=dt).element_size()
-        views.append(buf[o:o + nbytes].view(dt).view(shape))
-    return buf, views
+    return buf, _views(buf, specs)
 
 
 class DecodeStep:
@@ -89,8 +95,8 @@ class DecodeStep:
         # arena, so that a host-driven step is one copy in and one copy out
         self.in_arena, (self.q, self.ctx_lens, self.span_offsets, self.spans) = _arena(
             dev, [((B, H, D), dt), ((B,), torch.int32), ((B + 1,), torch.int32), ((max(len(spans), span_capacity), 2), torch.int32)])
-        self.out_arena, (self.out, self.lse, self.counts, self.status) = _arena(
-            dev, [((B, H, D), odt), ((B, H), torch.float32), ((B,), torch.int32), ((1,), torch.int32)])
+        self._out_specs = [((B, H, D), odt), ((B, H), torch.float32), ((B,), torch.int32), ((1,), torch.int32)]
+        self.out_arena, (self.out, self.lse, self.counts, self.status) = _arena(dev, self._out_specs)
         self.q.copy_(bits_to_tensor(wl.q_bits(), wl.dtype))
         self.ctx_lens.copy_(torch.from_numpy(wl.ctx_lens.copy()))
         self.span_offsets.copy_(torch.from_numpy(wl.span_offsets.copy()))
@@ -166,20 +172,34 @@ class DecodeStep:
         self._host_steps = {}
         self.h_in = self.in_arena.cpu().pin_memory()
         self.h_out = torch.empty(self.out_arena.shape, dtype=torch.uint8).pin_memory()
+        self.h_out_rows, self.h_lse, self.h_counts, self.h_status = _views(self.h_out, self._out_specs)
         return self.h_in.numel(), self.h_out.numel()
 
-    def step_from_host(self, stream=None):
+    def step_from_host(self, stream=None, direct=False):
         """Decode step whose per-step inputs start in pinned host memory and
         whose result ends there (ssa_decode_step with both copies); the KV
-        cache is the resident state."""
+        cache is the resident state.
+
+        direct=False: one copy-engine transfer in, the kernels, one out.
+        direct=True: the inputs are fetched by a kernel, the attention kernels
+        store output rows and lse straight into the pinned landing buffer, and
+        a kernel carries counts and the status word over
+        (SSA_STEP_COPY_BY_KERNEL).  Same bytes, same result, less latency."""
         if not hasattr(self, "h_in"):
             raise RuntimeError("call make_host_buffers() before step_from_host()")
-        key = (self.k.data_ptr(), self.max_selected)
+        key = (self.k.data_ptr(), self.max_selected, bool(direct))
         st = self._host_steps.get(key)
         if st is None:
-            st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q,
-                               self.k, self.v, self.max_selected, self.out, self.lse, self.workspace, self.status,
-                               host_in=self.h_in, dev_in=self.in_arena, host_out=self.h_out, dev_out=self.out_arena)
+            if direct:
+                tail = self.counts.data_ptr() - self.out_arena.data_ptr()   # counts + status: kernels read them too
+                st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q,
+                                   self.k, self.v, self.max_selected, self.h_out_rows, self.h_lse, self.workspace,
+                                   self.status, host_in=self.h_in, dev_in=self.in_arena,
+                                   host_out=self.h_out[tail:], dev_out=self.out_arena[tail:], copy_by_kernel=True)
+            else:
+                st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q,
+                                   self.k, self.v, self.max_selected, self.out, self.lse, self.workspace, self.status,
+                                   host_in=self.h_in, dev_in=self.in_arena, host_out=self.h_out, dev_out=self.out_arena)
             self._host_steps[key] = st
         return ssa.decode_step(self.desc, st, stream)
 

@@ -112,3 +112,24 @@ def test_error_raises_through_binding():
     with pytest.raises(ssa.SsaError) as e:
         ssa._check("ssa_decode_attn_sparse", ssa.ERR_WORKSPACE, True)
     assert "workspace" in str(e.value)
+
+
+def test_step_rejects_bad_copy_requests_before_enqueuing_anything():
+    d = good_desc()
+    st = ssa.Step()
+    assert ssa.lib.ssa_decode_step(None, C.byref(st), None) == ssa.ERR_NULL
+    st.host_in, st.dev_in, st.in_bytes = 0x1000, None, 256
+    assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_NULL         # a copy without a destination
+    st.dev_in = 0x2000
+    st.flags = 2
+    assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_UNSUPPORTED  # unknown flag bit
+    st.flags = ssa.STEP_COPY_BY_KERNEL
+    st.host_in = 0x1008
+    assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_ALIGN
+    st.host_in, st.in_bytes = 0x1000, 250
+    assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_ALIGN
+    import numpy as np
+    buf = np.zeros(4096 + 64, np.uint8)                                          # ordinary pageable memory
+    addr = (buf.ctypes.data + 63) // 64 * 64
+    st.host_in, st.in_bytes = addr, 256
+    assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_UNSUPPORTED  # kernels cannot address it

@@ -368,6 +368,49 @@ def test_decode_step_in_one_call_with_host_copies():
     assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_WORKSPACE
 
 
+@pytest.mark.parametrize("cfg,B,H", [(2, 5, 4), (3, 2, 4)])
+def test_decode_step_with_copies_done_by_kernels_and_rows_stored_into_host_memory(cfg, B, H):
+    # SSA_STEP_COPY_BY_KERNEL with out / lse pointing into the pinned landing buffer (one chunk per request
+    # at cfg 2, several plus the second pass at cfg 3): same bits as the device-resident step, and as the oracle
+    wl = inputs.make_config(cfg, B=B, H=H)
+    ds = DecodeStep(wl, out_dtype=torch.float32)
+    ds.step()
+    torch.cuda.synchronize()
+    want_out, want_lse, want_counts = ds.out.cpu(), ds.lse.cpu(), ds.counts.cpu()
+    ds.make_host_buffers()
+    for rep in range(2):                                       # twice: the second call overwrites the first
+        ds.in_arena.zero_()
+        ds.out_arena.fill_(7)
+        ds.status.zero_()
+        ds.h_out.fill_(9)
+        ds.index.fill_(-7)
+        before = ssa.launch_count()
+        ds.step_from_host(direct=True)
+        torch.cuda.synchronize()
+        assert ssa.launch_count() - before >= 4                # copy in, index, attention, copy out
+        assert torch.equal(ds.h_out_rows, want_out) and torch.equal(ds.h_lse, want_lse)
+        assert torch.equal(ds.h_counts, want_counts) and int(ds.h_status.item()) == 0
+        assert torch.equal(ds.in_arena.cpu(), ds.h_in)         # inputs arrived on the device
+        assert bool((ds.out.view(torch.uint8) == 7).all())     # the device-side output rows were not used
+    ref, _ = O.decode_attn_sparse(wl.q_bits(), *wl.kv_bits(), wl.ctx_lens,
+                                  *O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, ds.index_stride)[:2],
+                                  scale_of(wl.D), wl.dtype)
+    assert_parity(ds.h_out_rows.to(torch.float64).numpy(), ref, False, "direct to host")
+    # refusals come before anything is enqueued
+    pageable = torch.empty(ds.h_in.numel(), dtype=torch.uint8)
+    mk = lambda **kw: ssa.make_step(ds.span_offsets, ds.spans, ds.ctx_lens, ds.index, ds.counts, ds.q, ds.k, ds.v,
+                                    ds.max_selected, ds.out, ds.lse, ds.workspace, ds.status, **kw)
+    before = ssa.launch_count()
+    st = mk(host_in=pageable, dev_in=ds.in_arena, copy_by_kernel=True)
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_UNSUPPORTED      # not page-locked
+    st = mk(host_in=ds.h_in[8:264], dev_in=ds.in_arena, copy_by_kernel=True)
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_ALIGN
+    st = mk(host_in=ds.h_in, dev_in=ds.in_arena)
+    st.flags = 6
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_UNSUPPORTED      # unknown flag bits
+    assert ssa.launch_count() == before
+
+
 def test_side_stream_graph_replay_and_determinism():
     wl = inputs.make_config(3, B=2, H=4)
     ds = DecodeStep(wl, out_dtype=torch.float32)
