@@ -227,6 +227,23 @@ int32_t ssa_refs_to_spans(const ssa_anchor_tables* tables, int32_t B, int32_t* s
                           int32_t* spans_out, int32_t span_stride, uint32_t* dev_status, void* stream);
 
 /*
+ * ssa_refs_to_spans and ssa_spans_to_index in one launch (same passages of the
+ * paper): the lists index[b, 0 .. counts[b]) are exactly those the two calls
+ * produce with span_stride = SSA_MAX_SPANS_PER_SEQ, but the span list stays in
+ * shared memory.  The device status bits are those of the two calls
+ * (SSA_DEV_BAD_REF; SSA_DEV_BAD_SPAN / SSA_DEV_CLIPPED for lines, prefixes or
+ * current lines that do not fit the context; SSA_DEV_OVERFLOW for more than
+ * index_stride positions); a request that resolves to more than
+ * SSA_MAX_SPANS_PER_SEQ spans keeps the first ones
+ * (SSA_DEV_TOO_MANY_SPANS).  index, counts as for ssa_spans_to_index.
+ * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE (B <= 0, B > 65535, index_stride <= 0),
+ * SSA_ERR_ALIGN, SSA_ERR_CUDA.
+ */
+int32_t ssa_refs_to_index(const ssa_anchor_tables* tables, int32_t B, int32_t* index,
+                          int32_t index_stride, int32_t* counts, uint32_t* dev_status,
+                          void* stream);
+
+/*
  * The paper's own metadata format (Sec. "CUDA Kernel Design", Attention span
  * encoding): the context is cut into blocks of `block_size` positions; for
  * every block that holds at least one selected position the list records the

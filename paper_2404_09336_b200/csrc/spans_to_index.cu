@@ -14,7 +14,12 @@
 //      however uneven the spans are.
 // Blocks of one request repeat steps 1-3 (a few microseconds) instead of
 // communicating.
-#include "ssa_common.cuh"
+//
+// ssa_refs_to_index runs the same kernel with another step 1: one warp
+// resolves the request's references into spans (as ssa_refs_to_spans does) and
+// packs them straight into the keys in shared memory, so the span list never
+// goes through global memory and the step is one launch instead of two.
+#include "refs_resolve.cuh"
 
 namespace ssa {
 
@@ -22,39 +27,69 @@ constexpr int kIdxThreads = 128;
 constexpr int kMaxSpans = SSA_MAX_SPANS_PER_SEQ;   // power of two
 constexpr unsigned long long kEmptyKey = 0xffffffffffffffffull;
 
+// Where the spans of a request come from: a span list in global memory, or the anchor tables.
+struct SpanSource {
+  const int32_t* span_offsets;
+  const int32_t* spans;
+  const int32_t* ctx_lens;
+  ssa_anchor_tables tables;
+};
+
+template <bool kFromRefs>
 __global__ void __launch_bounds__(kIdxThreads)
-spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* __restrict__ spans,
-                      const int32_t* __restrict__ ctx_lens, int32_t* __restrict__ index,
+spans_to_index_kernel(const SpanSource src, int32_t* __restrict__ index,
                       int32_t index_stride, int32_t slice, int32_t* __restrict__ counts,
                       uint32_t* __restrict__ dev_status) {
   __shared__ unsigned long long keys[kMaxSpans];
   __shared__ int32_t new_start[kMaxSpans];
   __shared__ int32_t offs[kMaxSpans + 1];
   __shared__ uint32_t s_flags;
+  __shared__ int s_resolved;
+  const int32_t* __restrict__ span_offsets = src.span_offsets;
+  const int32_t* __restrict__ spans = src.spans;
+  const int32_t* __restrict__ ctx_lens = kFromRefs ? src.tables.ctx_lens : src.ctx_lens;
 
   const int b = blockIdx.y;
   const int tid = threadIdx.x;
   grid_dependency_wait();      // dependents are released when this grid completes: blocks of a large
                                // attention grid parked on the SMs during this kernel slowed it down
   const int n = max(ctx_lens[b], 0);
-  const int first = span_offsets[b];
-  int S = span_offsets[b + 1] - first;
   uint32_t flags = 0;
-  if (S < 0) S = 0;
-  if (S > kMaxSpans) { S = kMaxSpans; flags |= SSA_DEV_TOO_MANY_SPANS; }
-  int P = 32;
-  while (P < S) P <<= 1;
   if (tid == 0) s_flags = 0;
-  __syncthreads();
 
   // clamp a span to the context and pack it; empty spans get the sentinel
-  auto load_key = [&](int i) -> unsigned long long {
-    if (i >= S) return kEmptyKey;
-    const int2 se = reinterpret_cast<const int2*>(spans)[first + i];
+  auto pack = [&](int2 se) -> unsigned long long {
     if (se.x < 0 || se.x > se.y) flags |= SSA_DEV_BAD_SPAN;
     if (se.y > n) flags |= SSA_DEV_CLIPPED;
     const int s = max(se.x, 0), e = min(se.y, n);
     return e > s ? ((unsigned long long)(uint32_t)s << 32) | (uint32_t)e : kEmptyKey;
+  };
+
+  int first = 0, S;
+  if (kFromRefs) {
+    // 1 (references): warp 0 resolves them and leaves the packed spans, unsorted, in keys[0, S)
+    if (tid < 32) {
+      const int resolved = resolve_refs_warp(src.tables, b, tid, flags, [&](int at, int2 span) {
+        if (at < kMaxSpans) keys[at] = pack(span);
+      });
+      if (tid == 0) s_resolved = resolved;
+    }
+    __syncthreads();
+    S = s_resolved;
+  } else {
+    first = span_offsets[b];
+    S = span_offsets[b + 1] - first;
+  }
+  if (S < 0) S = 0;
+  if (S > kMaxSpans) { S = kMaxSpans; flags |= SSA_DEV_TOO_MANY_SPANS; }
+  int P = 32;
+  while (P < S) P <<= 1;
+  __syncthreads();
+
+  auto load_key = [&](int i) -> unsigned long long {
+    if (i >= S) return kEmptyKey;
+    if (kFromRefs) return keys[i];
+    return pack(reinterpret_cast<const int2*>(spans)[first + i]);
   };
 
   if (P == 32) {
@@ -62,6 +97,7 @@ spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* _
     // shuffles, no block barrier needed
     if (tid < 32) {
       const unsigned long long key = load_key(tid);
+      if (kFromRefs) __syncwarp();                  // every lane has read its key before any is overwritten
       int rank = 0;
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
@@ -72,8 +108,9 @@ spans_to_index_kernel(const int32_t* __restrict__ span_offsets, const int32_t* _
       __syncwarp();
     }
   } else {
-    // 1. load, clamp, pack
-    for (int i = tid; i < P; i += kIdxThreads) keys[i] = load_key(i);
+    // 1. load, clamp, pack (references: the keys are in place, only the padding is missing)
+    for (int i = tid; i < P; i += kIdxThreads)
+      if (!kFromRefs || i >= S) keys[i] = load_key(i);
     __syncthreads();
     // 2. bitonic sort, ascending by (start, end); empty keys sink to the end
     for (int k = 2; k <= P; k <<= 1) {
@@ -160,9 +197,32 @@ extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t
   if (slices > 32) slices = 32;
   const int32_t slice = (index_stride + slices - 1) / slices;
   dim3 grid((unsigned)slices, (unsigned)B);
-  const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel, grid, dim3(ssa::kIdxThreads),
-                                          (cudaStream_t)stream, span_offsets, spans, ctx_lens, index,
-                                          index_stride, slice, counts, dev_status);
+  ssa::SpanSource src = {};
+  src.span_offsets = span_offsets; src.spans = spans; src.ctx_lens = ctx_lens;
+  const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel<false>, grid, dim3(ssa::kIdxThreads),
+                                          (cudaStream_t)stream, src, index, index_stride, slice, counts,
+                                          dev_status);
+  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  ssa::note_launches(1);
+  return SSA_OK;
+}
+
+extern "C" int32_t ssa_refs_to_index(const ssa_anchor_tables* tables, int32_t B, int32_t* index,
+                                     int32_t index_stride, int32_t* counts, uint32_t* dev_status,
+                                     void* stream) {
+  if (!index || !counts) return SSA_ERR_NULL;
+  const int32_t rc = ssa::check_anchor_tables(tables);
+  if (rc != SSA_OK) return rc;
+  if (B <= 0 || B > 65535 || index_stride <= 0) return SSA_ERR_SHAPE;
+  int slices = (index_stride + 511) / 512;
+  if (slices > 32) slices = 32;
+  const int32_t slice = (index_stride + slices - 1) / slices;
+  dim3 grid((unsigned)slices, (unsigned)B);
+  ssa::SpanSource src = {};
+  src.tables = *tables;
+  const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel<true>, grid, dim3(ssa::kIdxThreads),
+                                          (cudaStream_t)stream, src, index, index_stride, slice, counts,
+                                          dev_status);
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   ssa::note_launches(1);
   return SSA_OK;

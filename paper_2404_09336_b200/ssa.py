@@ -83,6 +83,8 @@ def _load():
                                               C.c_int32, vp, vp, vp, C.c_size_t, vp, vp]
     lib.ssa_refs_to_spans.restype = C.c_int32
     lib.ssa_refs_to_spans.argtypes = [C.POINTER(AnchorTables), C.c_int32, vp, vp, C.c_int32, vp, vp]
+    lib.ssa_refs_to_index.restype = C.c_int32
+    lib.ssa_refs_to_index.argtypes = [C.POINTER(AnchorTables), C.c_int32, vp, C.c_int32, vp, vp, vp]
     lib.ssa_decode_step.restype = C.c_int32
     lib.ssa_decode_step.argtypes = [C.POINTER(AttnDesc), C.POINTER(Step), vp]
     lib.ssa_decode_attn_sparse_noalloc.restype = C.c_int32
@@ -208,14 +210,31 @@ def decode_attn_blockmask(desc, q, k_cache, v_cache, ctx_lens, block_idx, block_
     return _check("ssa_decode_attn_blockmask", rc, check)
 
 
-def refs_to_spans(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
-                  ctx_lens, span_offsets_out, spans_out, dev_status=None, stream=None, check=True):
-    """ssa_refs_to_spans: spans_out[B, span_stride, 2] and span_offsets_out[B+1] are written."""
+def _anchor_tables(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
+                   ctx_lens) -> AnchorTables:
     t = AnchorTables()
     for name, ten in (("line_offsets", line_offsets), ("lines", lines), ("anchor_offsets", anchor_offsets),
                       ("anchor_line", anchor_line), ("ref_offsets", ref_offsets), ("refs", refs),
                       ("prefix_len", prefix_len), ("line_start", line_start), ("ctx_lens", ctx_lens)):
         setattr(t, name, None if ten is None else ten.data_ptr())
+    return t
+
+
+def refs_to_index(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
+                  ctx_lens, index, counts, dev_status=None, stream=None, check=True):
+    """ssa_refs_to_index: references -> index[B, index_stride] and counts[B] in one launch."""
+    t = _anchor_tables(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
+                       ctx_lens)
+    rc = lib.ssa_refs_to_index(C.byref(t), int(ctx_lens.numel()), _ptr(index), _row_stride(index), _ptr(counts),
+                               _ptr(dev_status), _stream(stream))
+    return _check("ssa_refs_to_index", rc, check)
+
+
+def refs_to_spans(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
+                  ctx_lens, span_offsets_out, spans_out, dev_status=None, stream=None, check=True):
+    """ssa_refs_to_spans: spans_out[B, span_stride, 2] and span_offsets_out[B+1] are written."""
+    t = _anchor_tables(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
+                       ctx_lens)
     rc = lib.ssa_refs_to_spans(C.byref(t), int(ctx_lens.numel()), _ptr(span_offsets_out), _ptr(spans_out),
                                int(spans_out.shape[1]), _ptr(dev_status), _stream(stream))
     return _check("ssa_refs_to_spans", rc, check)

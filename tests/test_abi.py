@@ -133,3 +133,20 @@ def test_step_rejects_bad_copy_requests_before_enqueuing_anything():
     addr = (buf.ctypes.data + 63) // 64 * 64
     st.host_in, st.in_bytes = addr, 256
     assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_UNSUPPORTED  # kernels cannot address it
+
+
+def test_refs_to_index_rejects_bad_arguments():
+    t = ssa.AnchorTables()
+    for name, _ in t._fields_:
+        setattr(t, name, 0x1000)
+    call = lambda tab, B, index, stride, counts: ssa.lib.ssa_refs_to_index(
+        C.byref(tab) if tab is not None else None, B, index, stride, counts, None, None)
+    assert call(None, 1, 0x2000, 64, 0x3000) == ssa.ERR_NULL
+    assert call(t, 1, None, 64, 0x3000) == ssa.ERR_NULL
+    assert call(t, 0, 0x2000, 64, 0x3000) == ssa.ERR_SHAPE
+    assert call(t, 70000, 0x2000, 64, 0x3000) == ssa.ERR_SHAPE
+    assert call(t, 1, 0x2000, 0, 0x3000) == ssa.ERR_SHAPE
+    t.refs = 0x1004
+    assert call(t, 1, 0x2000, 64, 0x3000) == ssa.ERR_ALIGN
+    t.refs, t.lines = 0x1000, None
+    assert call(t, 1, 0x2000, 64, 0x3000) == ssa.ERR_NULL

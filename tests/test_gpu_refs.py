@@ -1,4 +1,5 @@
-"""ssa_refs_to_spans against the oracle (bit-exact span rows), and the whole
+"""ssa_refs_to_spans against the oracle (bit-exact span rows), ssa_refs_to_index
+(the same plus the index expansion in one launch, bit-exact lists), and the whole
 chain references -> spans -> index lists -> attention on the device."""
 import random
 
@@ -52,25 +53,7 @@ def compare(reqs, stride):
     return so, sp, ctx
 
 
-def test_paper_examples_and_flags():
-    arith = dict(lines=[(0, 14), (14, 40), (40, 54), (54, 66)], anchors=[0, 2, 3], refs=[(0, 0), (1, 1), (2, 2)],
-                 prefix=0, start=66, ctx=69)
-    summ = dict(lines=[(12 + 8 * i, 20 + 8 * i) for i in range(31)] + [(260, 280)], anchors=list(range(31)),
-                refs=[(17, 19), (-1, -1)], prefix=12, start=280, ctx=291)
-    so, sp, ctx = compare([arith, summ], 8)
-    # union of the resolved spans = the positions the paper's examples attend to
-    assert O.spans_to_index(sp[0].cpu().numpy(), 69).tolist() == list(range(0, 14)) + list(range(40, 69))
-    assert O.spans_to_index(sp[1].cpu().numpy(), 291).tolist() == \
-        list(range(0, 12)) + list(range(148, 172)) + list(range(260, 291))
-    compare([dict(arith, refs=[(0, 2), (-1, -1), (-2, -2), (-4, -4)])], 5)          # overflow: 2 + 6 spans
-    for bad in ([(5, 5)], [(-9, -9)], [(1, 0)], [(-1, 2)], [(0, 7)]):
-        compare([dict(arith, refs=bad)], 8)
-    compare([dict(lines=[], anchors=[], refs=[], prefix=3, start=3, ctx=9)], 2)
-    compare([dict(arith, anchors=[0, 9, 3])], 8)                                    # an anchor that points nowhere
-
-
-@pytest.mark.parametrize("seed", range(5))
-def test_fuzz(seed):
+def fuzz_requests(seed):
     rnd = random.Random(seed)
     reqs = []
     for _ in range(rnd.randint(1, 30)):
@@ -91,7 +74,96 @@ def test_fuzz(seed):
                 a = rnd.randint(-1, len(anchors) + 1)
                 refs.append((a, a + rnd.randint(-1, 4)))
         reqs.append(dict(lines=lines, anchors=anchors, refs=refs, prefix=prefix, start=pos, ctx=pos + rnd.randint(0, 9)))
-    compare(reqs, rnd.choice([4, 32, 100]))
+    return reqs
+
+
+def run_refs_index(reqs, index_stride):
+    B = len(reqs)
+    lo, ld = flat([r["lines"] for r in reqs], 2)
+    ao, ad = flat([[(a,) for a in r["anchors"]] for r in reqs], 1)
+    ro, rd = flat([r["refs"] for r in reqs], 2)
+    i32 = lambda k: torch.tensor([r[k] for r in reqs], dtype=torch.int32, device=DEV)
+    index = torch.full((B, index_stride), -7, dtype=torch.int32, device=DEV)
+    counts = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ssa.refs_to_index(lo, ld, ao, ad.view(-1), ro, rd, i32("prefix"), i32("start"), i32("ctx"), index, counts, status)
+    torch.cuda.synchronize()
+    return index.cpu().numpy(), counts.cpu().numpy(), int(status.item())
+
+
+def compare_index(reqs, index_stride, max_spans=2048):
+    """One launch against the oracle's resolver followed by its span -> index definition."""
+    index, counts, status = run_refs_index(reqs, index_stride)
+    want_status = 0
+    for b, r in enumerate(reqs):
+        spans, st = O.resolve_references(r["lines"], r["anchors"], r["refs"], r["prefix"], r["start"], r["ctx"])
+        if len(spans) > max_spans:
+            spans, st = spans[:max_spans], st | 1 << 20          # marker for "too many spans"
+        want_status |= st | O.spans_status(spans, r["ctx"], index_stride)
+        idx = O.spans_to_index(spans, r["ctx"])[:index_stride]
+        assert counts[b] == len(idx), f"request {b}"
+        assert index[b, :len(idx)].tolist() == idx.tolist(), f"request {b}"
+        assert np.all(index[b, len(idx):] == -7)                 # nothing written past the list
+    gpu_bits = {O.ST_BAD_SPAN: ssa.DEV_BAD_SPAN, O.ST_CLIPPED: ssa.DEV_CLIPPED, O.ST_OVERFLOW: ssa.DEV_OVERFLOW,
+                O.ST_BAD_REF: ssa.DEV_BAD_REF, 1 << 20: ssa.DEV_TOO_MANY_SPANS}
+    assert status == sum(v for k, v in gpu_bits.items() if want_status & k)
+    return index, counts
+
+
+def test_paper_examples_and_flags():
+    arith = dict(lines=[(0, 14), (14, 40), (40, 54), (54, 66)], anchors=[0, 2, 3], refs=[(0, 0), (1, 1), (2, 2)],
+                 prefix=0, start=66, ctx=69)
+    summ = dict(lines=[(12 + 8 * i, 20 + 8 * i) for i in range(31)] + [(260, 280)], anchors=list(range(31)),
+                refs=[(17, 19), (-1, -1)], prefix=12, start=280, ctx=291)
+    so, sp, ctx = compare([arith, summ], 8)
+    # union of the resolved spans = the positions the paper's examples attend to
+    assert O.spans_to_index(sp[0].cpu().numpy(), 69).tolist() == list(range(0, 14)) + list(range(40, 69))
+    assert O.spans_to_index(sp[1].cpu().numpy(), 291).tolist() == \
+        list(range(0, 12)) + list(range(148, 172)) + list(range(260, 291))
+    compare([dict(arith, refs=[(0, 2), (-1, -1), (-2, -2), (-4, -4)])], 5)          # overflow: 2 + 6 spans
+    for bad in ([(5, 5)], [(-9, -9)], [(1, 0)], [(-1, 2)], [(0, 7)]):
+        compare([dict(arith, refs=bad)], 8)
+    compare([dict(lines=[], anchors=[], refs=[], prefix=3, start=3, ctx=9)], 2)
+    compare([dict(arith, anchors=[0, 9, 3])], 8)                                    # an anchor that points nowhere
+
+
+def test_one_launch_paper_examples_and_flags():
+    arith = dict(lines=[(0, 14), (14, 40), (40, 54), (54, 66)], anchors=[0, 2, 3], refs=[(0, 0), (1, 1), (2, 2)],
+                 prefix=0, start=66, ctx=69)
+    summ = dict(lines=[(12 + 8 * i, 20 + 8 * i) for i in range(31)] + [(260, 280)], anchors=list(range(31)),
+                refs=[(17, 19), (-1, -1)], prefix=12, start=280, ctx=291)
+    index, counts = compare_index([arith, summ], 320)
+    assert index[0, :counts[0]].tolist() == list(range(0, 14)) + list(range(40, 69))
+    assert index[1, :counts[1]].tolist() == list(range(0, 12)) + list(range(148, 172)) + list(range(260, 291))
+    compare_index([arith, summ], 40)                                                # lists cut at index_stride
+    for bad in ([(5, 5)], [(-9, -9)], [(1, 0)], [(-1, 2)], [(0, 7)]):
+        compare_index([dict(arith, refs=bad)], 96)
+    compare_index([dict(lines=[], anchors=[], refs=[], prefix=3, start=3, ctx=9)], 16)
+    compare_index([dict(arith, anchors=[0, 9, 3])], 96)                             # an anchor that points nowhere
+    compare_index([dict(arith, ctx=60)], 96)                                        # lines beyond the context: clipped
+    compare_index([dict(arith, prefix=-2), dict(arith, start=80)], 96)              # malformed prefix / current line
+    # many references: more than 32 spans (sorted in shared memory by the whole block), and more than the
+    # 2048 a request may resolve to (the first 2048 are kept)
+    lines = [(4 * i, 4 * i + 3) for i in range(700)]
+    many = dict(lines=lines, anchors=list(range(700)), refs=[(i, i + 2) for i in range(0, 690, 7)], prefix=0,
+                start=2800, ctx=2810)
+    compare_index([many, arith], 2816)
+    too_many = dict(many, refs=[(0, 699)] * 3)
+    compare_index([too_many, summ], 2816)
+    # several output slices per request
+    compare_index([dict(many, refs=[(0, 699)])], 2816)
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_one_launch_fuzz(seed):
+    reqs = fuzz_requests(seed + 100)
+    compare_index(reqs, random.Random(seed).choice([64, 700, 2000]))
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_fuzz(seed):
+    reqs = fuzz_requests(seed)
+    compare(reqs, random.Random(seed + 50).choice([4, 32, 100]))
 
 
 def test_references_to_attention_on_the_device():
