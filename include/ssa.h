@@ -187,6 +187,46 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q,
                               uint32_t* dev_status, void* stream);
 
 /*
+ * The two attention calls over a PAGED cache (the paper pre-allocates one
+ * contiguous cache per request, Experimental results; paging has no
+ * counterpart there - it is what serving stacks use to avoid that
+ * reservation).  K and V live in pools of n_pages pages of page_size rows;
+ * logical position t of request b is pool row
+ *     page_table[b * page_table_stride + t / page_size] * page_size + t % page_size,
+ * whose head h starts at pool + row * k_stride_t + (h / (H/H_kv)) * k_stride_h
+ * elements (desc->k_stride_b / v_stride_b are ignored; a pool laid out
+ * [n_pages, page_size, H_kv, D] has k_stride_t = H_kv*D, k_stride_h = D).
+ * desc->max_ctx bounds the logical context.  Everything else - index lists,
+ * counts, results, workspace size, status bits - is as for
+ * ssa_decode_attn_sparse / ssa_decode_attn_dense; a page-table entry outside
+ * [0, n_pages) makes the positions it covers be skipped (SSA_DEV_BAD_INDEX).
+ * The position -> row translation happens once per block, while it stages its
+ * list entries, and costs one extra page-table read per entry.
+ *   page_table  dev int32 [B * page_table_stride]
+ * Errors as for the unpaged calls, plus SSA_ERR_NULL for a missing paging
+ * struct or table and SSA_ERR_SHAPE for page_size not a power of two,
+ * n_pages <= 0, n_pages * page_size >= 2^31 or
+ * page_table_stride * page_size < desc->max_ctx.
+ */
+typedef struct {
+  const int32_t* page_table;
+  int32_t page_table_stride;   /* entries per request */
+  int32_t page_size;           /* rows per page, a power of two */
+  int32_t n_pages;             /* pages in the pool */
+} ssa_paging;
+
+int32_t ssa_decode_attn_sparse_paged(const ssa_attn_desc* desc, const void* q, const void* k_pool,
+                                     const void* v_pool, const ssa_paging* paging,
+                                     const int32_t* ctx_lens, const int32_t* index,
+                                     int32_t index_stride, const int32_t* counts,
+                                     int32_t max_selected, void* out, float* lse, void* workspace,
+                                     size_t workspace_bytes, uint32_t* dev_status, void* stream);
+int32_t ssa_decode_attn_dense_paged(const ssa_attn_desc* desc, const void* q, const void* k_pool,
+                                    const void* v_pool, const ssa_paging* paging,
+                                    const int32_t* ctx_lens, void* out, float* lse, void* workspace,
+                                    size_t workspace_bytes, uint32_t* dev_status, void* stream);
+
+/*
  * Anchors and references -> span lists: the step before ssa_spans_to_index
  * (Sec. "Self-selected attention span": anchors identify groups of contiguous
  * tokens, the model names the anchors it needs, generation attends to the

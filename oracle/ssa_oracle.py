@@ -418,3 +418,28 @@ def decode_attn_dense(q, k_cache, v_cache, ctx_lens, scale,
             out[b, h] = o
             lse[b, h] = e
     return out, lse
+
+
+def gather_pages(pool, page_table, page_size: int, max_ctx: int) -> np.ndarray:
+    """The contiguous cache [B, H, max_ctx, D] that a paged cache stands for.
+
+    ``pool`` [n_pages, page_size, H, D]; ``page_table`` [B, pages per request].
+    Logical position t of request b is row t % page_size of page
+    page_table[b, t // page_size].  (The paper pre-allocates a contiguous cache
+    per request, so paging has no passage there; this is only the definition of
+    the layout, after which the attention definitions above apply unchanged.)
+    Positions whose page id lies outside the pool are left zero; a test must not
+    select them when it compares with this function's result.
+    """
+    pool = np.asarray(pool)
+    page_table = np.asarray(page_table)
+    B = page_table.shape[0]
+    n_pages, ps, H, D = pool.shape
+    assert ps == page_size
+    cache = np.zeros((B, H, max_ctx, D), dtype=pool.dtype)
+    for b in range(B):
+        for t in range(max_ctx):
+            page = int(page_table[b, t // page_size])
+            if 0 <= page < n_pages:
+                cache[b, :, t, :] = pool[page, t % page_size]
+    return cache

@@ -62,6 +62,10 @@ struct DecodeParams {
   uint32_t k_row_bytes, v_row_bytes;   // token stride of the cache in bytes
   int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32, early_release;
   int32_t kv_group;         // query heads per K/V head (1: multi-head attention)
+  // paged cache (page_table != nullptr): logical position t of request b is row
+  // page_table[b * page_table_stride + (t >> page_shift)] << page_shift | (t & page_mask) of the pool
+  const int32_t* page_table;
+  int32_t page_table_stride, page_shift, page_mask, n_pages;
   float scale_log2;         // softmax scale * log2(e)
 };
 
@@ -145,11 +149,11 @@ decode_partial_kernel(const DecodeParams p) {
   };
   int32_t raw[kIdxPerThread];
   if (kMode == kIndex) {
-    const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
+    const int32_t* row = p.index ? p.index + (int64_t)b * p.index_stride + start : nullptr;   // null: 0, 1, 2, ...
 #pragma unroll
     for (int j = 0; j < kIdxPerThread; ++j) {
       const int r = staged_row(lane + 32 * j);
-      raw[j] = (r < p.chunk && start + r < p.max_selected) ? __ldg(row + r) : -1;
+      raw[j] = (r < p.chunk && start + r < p.max_selected) ? (p.index ? __ldg(row + r) : start + r) : -1;
     }
   }
   Piece qraw;
@@ -202,7 +206,13 @@ decode_partial_kernel(const DecodeParams p) {
       const int r = staged_row(lane + 32 * j);
       if (r < cnt) {
         int v = raw[j];
-        if (v < 0 || v >= n) { v = -1; flags |= SSA_DEV_BAD_INDEX; bad = true; }
+        if (v < 0 || v >= n) {
+          v = -1; flags |= SSA_DEV_BAD_INDEX; bad = true;
+        } else if (p.page_table) {                    // logical position -> row of the pool
+          const int page = __ldg(p.page_table + (int64_t)b * p.page_table_stride + (v >> p.page_shift));
+          if ((unsigned)page < (unsigned)p.n_pages) v = (page << p.page_shift) | (v & p.page_mask);
+          else { v = -1; flags |= SSA_DEV_BAD_INDEX; bad = true; }
+        }
         s_idx[r] = v;
       }
     }
@@ -443,14 +453,28 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
                    const int32_t* ctx_lens, const int32_t* index, int32_t index_stride,
                    const int32_t* counts, int32_t max_selected, void* out, float* lse,
                    void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream, int mode,
-                   const BlockList* bl = nullptr) {
+                   const BlockList* bl = nullptr, const ssa_paging* pg = nullptr) {
+  // a paged cache is read through the staged-positions path; without a list the positions are 0 .. ctx_len-1
+  const bool dense_paged = pg && mode == kDense;
+  if (dense_paged) mode = kIndex;
   const bool sparse = mode == kIndex;
   if (!d || !q || !k || !v || !ctx_lens || !out) return SSA_ERR_NULL;
-  if (sparse && (!index || !counts)) return SSA_ERR_NULL;
+  if (sparse && !dense_paged && (!index || !counts)) return SSA_ERR_NULL;
+  if (pg) {
+    if (!pg->page_table) return SSA_ERR_NULL;
+    if (mode == kBlockMask) return SSA_ERR_UNSUPPORTED;
+    if (pg->page_size <= 0 || (pg->page_size & (pg->page_size - 1)) != 0 || pg->n_pages <= 0 ||
+        pg->page_table_stride <= 0 || (long long)pg->n_pages * pg->page_size > 0x7fffffffll ||
+        (long long)pg->page_table_stride * pg->page_size < d->max_ctx)
+      return SSA_ERR_SHAPE;
+  }
   if (mode == kBlockMask && (!bl || !bl->block_idx || !bl->block_mask || !counts)) return SSA_ERR_NULL;
   const int32_t rc = check_desc(d);
   if (rc != SSA_OK) return rc;
-  if (mode != kDense) {
+  if (dense_paged) {
+    max_selected = d->max_ctx;
+    index_stride = d->max_ctx;
+  } else if (mode != kDense) {
     if (index_stride <= 0 || max_selected <= 0 || max_selected > index_stride) return SSA_ERR_CAPACITY;
   } else {
     max_selected = d->max_ctx;
@@ -469,8 +493,14 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   DecodeParams p;
   p.q = q; p.k = k; p.v = v;
   p.ctx_lens = ctx_lens;
-  p.index = sparse ? index : nullptr;
-  p.counts = mode != kDense ? counts : nullptr;
+  p.index = sparse && !dense_paged ? index : nullptr;
+  p.counts = mode != kDense && !dense_paged ? counts : nullptr;
+  p.page_table = pg ? pg->page_table : nullptr;
+  p.page_table_stride = pg ? pg->page_table_stride : 0;
+  p.n_pages = pg ? pg->n_pages : 0;
+  p.page_mask = pg ? pg->page_size - 1 : 0;
+  p.page_shift = 0;
+  while (pg && (1 << p.page_shift) < pg->page_size) ++p.page_shift;
   p.block_idx = mode == kBlockMask ? bl->block_idx : nullptr;
   p.block_mask = mode == kBlockMask ? bl->block_mask : nullptr;
   p.block_size = mode == kBlockMask ? bl->block_size : 0;
@@ -481,8 +511,8 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   p.dev_status = dev_status;
   p.q_sb = d->q_stride_b; p.q_sh = d->q_stride_h;
   p.kv_group = d->H / d->H_kv;
-  p.k_sb = d->k_stride_b; p.k_sh = d->k_stride_h;
-  p.v_sb = d->v_stride_b; p.v_sh = d->v_stride_h;
+  p.k_sb = pg ? 0 : d->k_stride_b; p.k_sh = d->k_stride_h;      // a pool has no batch dimension
+  p.v_sb = pg ? 0 : d->v_stride_b; p.v_sh = d->v_stride_h;
   p.k_row_bytes = (uint32_t)(d->k_stride_t * 2);
   p.v_row_bytes = (uint32_t)(d->v_stride_t * 2);
   p.o_sb = d->o_stride_b; p.o_sh = d->o_stride_h;
@@ -499,8 +529,8 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
 
   // one 256-bit load per lane needs every cache row piece on a 32-byte boundary
   const bool a32 = reinterpret_cast<uintptr_t>(k) % 32 == 0 && reinterpret_cast<uintptr_t>(v) % 32 == 0 &&
-                   d->k_stride_b % 16 == 0 && d->k_stride_t % 16 == 0 && d->k_stride_h % 16 == 0 &&
-                   d->v_stride_b % 16 == 0 && d->v_stride_t % 16 == 0 && d->v_stride_h % 16 == 0;
+                   p.k_sb % 16 == 0 && d->k_stride_t % 16 == 0 && d->k_stride_h % 16 == 0 &&
+                   p.v_sb % 16 == 0 && d->v_stride_t % 16 == 0 && d->v_stride_h % 16 == 0;
   cudaStream_t st = (cudaStream_t)stream;
   if (d->kv_dtype == SSA_BF16)
     return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, mode, a32, st)
@@ -584,6 +614,25 @@ int32_t ssa_decode_attn_dense(const ssa_attn_desc* desc, const void* q, const vo
                               void* stream) {
   return ssa::run(desc, q, k_cache, v_cache, ctx_lens, nullptr, 0, nullptr, 0, out, lse, workspace,
                   workspace_bytes, dev_status, stream, ssa::kDense);
+}
+
+int32_t ssa_decode_attn_sparse_paged(const ssa_attn_desc* desc, const void* q, const void* k_pool,
+                                     const void* v_pool, const ssa_paging* paging, const int32_t* ctx_lens,
+                                     const int32_t* index, int32_t index_stride, const int32_t* counts,
+                                     int32_t max_selected, void* out, float* lse, void* workspace,
+                                     size_t workspace_bytes, uint32_t* dev_status, void* stream) {
+  if (!paging) return SSA_ERR_NULL;
+  return ssa::run(desc, q, k_pool, v_pool, ctx_lens, index, index_stride, counts, max_selected, out, lse,
+                  workspace, workspace_bytes, dev_status, stream, ssa::kIndex, nullptr, paging);
+}
+
+int32_t ssa_decode_attn_dense_paged(const ssa_attn_desc* desc, const void* q, const void* k_pool,
+                                    const void* v_pool, const ssa_paging* paging, const int32_t* ctx_lens,
+                                    void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                    uint32_t* dev_status, void* stream) {
+  if (!paging) return SSA_ERR_NULL;
+  return ssa::run(desc, q, k_pool, v_pool, ctx_lens, nullptr, 0, nullptr, 0, out, lse, workspace,
+                  workspace_bytes, dev_status, stream, ssa::kDense, nullptr, paging);
 }
 
 }  // extern "C"

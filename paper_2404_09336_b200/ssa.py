@@ -49,6 +49,12 @@ class Step(C.Structure):
     ]
 
 
+class Paging(C.Structure):
+    """ssa_paging (see include/ssa.h)."""
+    _fields_ = [("page_table", C.c_void_p), ("page_table_stride", C.c_int32), ("page_size", C.c_int32),
+                ("n_pages", C.c_int32)]
+
+
 class AnchorTables(C.Structure):
     """ssa_anchor_tables (see include/ssa.h)."""
     _fields_ = [(n, C.c_void_p) for n in ("line_offsets", "lines", "anchor_offsets", "anchor_line", "ref_offsets",
@@ -83,6 +89,12 @@ def _load():
                                               C.c_int32, vp, vp, vp, C.c_size_t, vp, vp]
     lib.ssa_refs_to_spans.restype = C.c_int32
     lib.ssa_refs_to_spans.argtypes = [C.POINTER(AnchorTables), C.c_int32, vp, vp, C.c_int32, vp, vp]
+    lib.ssa_decode_attn_sparse_paged.restype = C.c_int32
+    lib.ssa_decode_attn_sparse_paged.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, C.POINTER(Paging), vp, vp, C.c_int32,
+                                                 vp, C.c_int32, vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_attn_dense_paged.restype = C.c_int32
+    lib.ssa_decode_attn_dense_paged.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, C.POINTER(Paging), vp, vp, vp, vp,
+                                                C.c_size_t, vp, vp]
     lib.ssa_refs_to_index.restype = C.c_int32
     lib.ssa_refs_to_index.argtypes = [C.POINTER(AnchorTables), C.c_int32, vp, C.c_int32, vp, vp, vp]
     lib.ssa_decode_step.restype = C.c_int32
@@ -208,6 +220,57 @@ def decode_attn_blockmask(desc, q, k_cache, v_cache, ctx_lens, block_idx, block_
                                        int(block_size), int(max_blocks), _ptr(out), _ptr(lse), _ptr(workspace),
                                        ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_blockmask", rc, check)
+
+
+def make_desc_paged(q, k_pool, v_pool, out, max_ctx: int, scale: float = 0.0) -> AttnDesc:
+    """Descriptor for q[B,H,D], out[B,H,D] and K/V pools [n_pages, page_size, H_kv, D] whose rows are evenly
+    spaced over the whole pool (pages back to back)."""
+    B, H, D = q.shape
+    d = AttnDesc()
+    d.B, d.H, d.H_kv, d.D = B, H, k_pool.shape[2], D
+    d.max_ctx = int(max_ctx)
+    d.kv_dtype = _DTYPES.get(k_pool.dtype, -1)
+    d.out_dtype = _DTYPES.get(out.dtype, -1)
+    d.scale = float(scale)
+    d.q_stride_b, d.q_stride_h = q.stride(0), q.stride(1)
+    d.o_stride_b, d.o_stride_h = out.stride(0), out.stride(1)
+    for pool in (k_pool, v_pool):
+        if pool.stride(-1) != 1 or pool.stride(0) != pool.shape[1] * pool.stride(1):
+            raise ValueError("pool rows must be evenly spaced and the head dimension contiguous")
+    d.k_stride_b = d.v_stride_b = 0
+    d.k_stride_t, d.k_stride_h = k_pool.stride(1), k_pool.stride(2)
+    d.v_stride_t, d.v_stride_h = v_pool.stride(1), v_pool.stride(2)
+    return d
+
+
+def make_paging(page_table, page_size: int, n_pages: int) -> Paging:
+    """ssa_paging for page_table[B, pages per request] (int32, device); keep the tensor alive."""
+    pg = Paging()
+    pg.page_table, pg.page_table_stride = page_table.data_ptr(), _row_stride(page_table)
+    pg.page_size, pg.n_pages = int(page_size), int(n_pages)
+    return pg
+
+
+def decode_attn_sparse_paged(desc, q, k_pool, v_pool, paging, ctx_lens, index, counts, max_selected, out, lse=None,
+                             workspace=None, dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_sparse_paged: as decode_attn_sparse over a paged cache."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_sparse_paged(C.byref(desc), _ptr(q), _ptr(k_pool), _ptr(v_pool),
+                                          C.byref(paging) if paging is not None else None, _ptr(ctx_lens),
+                                          _ptr(index), _row_stride(index) if index is not None else 0, _ptr(counts),
+                                          int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes,
+                                          _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_sparse_paged", rc, check)
+
+
+def decode_attn_dense_paged(desc, q, k_pool, v_pool, paging, ctx_lens, out, lse=None, workspace=None,
+                            dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_dense_paged: full-context attention over a paged cache."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_dense_paged(C.byref(desc), _ptr(q), _ptr(k_pool), _ptr(v_pool),
+                                         C.byref(paging) if paging is not None else None, _ptr(ctx_lens), _ptr(out),
+                                         _ptr(lse), _ptr(workspace), ws_bytes, _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_dense_paged", rc, check)
 
 
 def _anchor_tables(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets, refs, prefix_len, line_start,
