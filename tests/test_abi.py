@@ -150,3 +150,46 @@ def test_refs_to_index_rejects_bad_arguments():
     assert call(t, 1, 0x2000, 64, 0x3000) == ssa.ERR_ALIGN
     t.refs, t.lines = 0x1000, None
     assert call(t, 1, 0x2000, 64, 0x3000) == ssa.ERR_NULL
+
+
+def test_header_is_plain_c_and_cpp(tmp_path):
+    # the boundary is a C ABI: the header must compile as C99 and as C++ with nothing but the standard headers
+    import shutil
+    import subprocess
+    src = tmp_path / "use_ssa.c"
+    src.write_text('#include "ssa.h"\n'
+                   "int main(void) {\n"
+                   "  ssa_attn_desc d; ssa_step s; ssa_anchor_tables t; ssa_paging p;\n"
+                   "  (void)d; (void)s; (void)t; (void)p;\n"
+                   "  return (int)(sizeof(ssa_step) == 0) + (SSA_MAX_SPANS_PER_SEQ != 2048);\n"
+                   "}\n")
+    inc = os.path.join(ROOT, "include")
+    for cc, std in (("gcc", "-std=c99"), ("g++", "-std=c++11")):
+        exe = shutil.which(cc)
+        if exe is None:
+            pytest.skip(f"{cc} not installed")
+        args = [exe, std, "-Wall", "-Werror", "-pedantic", "-I", inc, "-fsyntax-only"]
+        args += ["-x", "c++"] if cc == "g++" else []
+        res = subprocess.run(args + [str(src)], capture_output=True, text=True)
+        assert res.returncode == 0, res.stderr
+
+
+def test_struct_layouts_of_the_binding_match_the_header(tmp_path):
+    # sizes and a few offsets of the ctypes mirrors against what the C compiler lays out
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("gcc not installed")
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "ssa.h"\n'
+                   "int main(void) {\n"
+                   '  printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(ssa_attn_desc), sizeof(ssa_step),\n'
+                   "         sizeof(ssa_anchor_tables), sizeof(ssa_paging), offsetof(ssa_attn_desc, scale),\n"
+                   "         offsetof(ssa_step, flags), offsetof(ssa_step, host_in), offsetof(ssa_paging, n_pages));\n"
+                   "  return 0;\n}\n")
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    got = [int(x) for x in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
+    want = [C.sizeof(ssa.AttnDesc), C.sizeof(ssa.Step), C.sizeof(ssa.AnchorTables), C.sizeof(ssa.Paging),
+            ssa.AttnDesc.scale.offset, ssa.Step.flags.offset, ssa.Step.host_in.offset, ssa.Paging.n_pages.offset]
+    assert got == want
