@@ -361,15 +361,29 @@ decode_merge_kernel(const DecodeParams p) {
   if (d == 0 && p.lse) p.lse[(int64_t)b * p.H + h] = L > 0.f ? (M + log2f(L)) * kLn2 : neg_inf();
 }
 
+}  // namespace ssa
+
+#include "decode_gqa.cuh"
+
+namespace ssa {
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 struct Plan { int chunk, n_chunks; size_t acc_bytes, total_bytes; };
 
+// Grouped query heads go to the kernel that reads a K/V row once for the whole group.
+static bool shares_rows(const ssa_attn_desc* d) {
+  const int group = d->H_kv > 0 ? d->H / d->H_kv : 1;
+  return d->D == 128 && group >= 2 && group <= kGqaHeads;
+}
+
 static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   if (!d || d->B <= 0 || d->H <= 0 || max_selected <= 0) return false;
   if (d->D != 64 && d->D != 128) return false;
-  const long long units = (long long)d->B * d->H;
+  const long long out_units = (long long)d->B * d->H;                  // triples per chunk
+  const long long units = shares_rows(d) ? (long long)d->B * d->H_kv   // blocks per chunk
+                                         : out_units;
   // The second pass costs about as much as two rounds of a block, so a request is split only when that buys
   // parallelism: one chunk whenever the list fits a block's staging area and either every SM gets a block or
   // the list is short anyway; otherwise 256-entry chunks, halved while the grid has under two blocks per SM.
@@ -381,8 +395,8 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   if (n_chunks == 1) chunk = (max_selected + 31) / 32 * 32;
   pl->chunk = chunk;
   pl->n_chunks = n_chunks;
-  pl->acc_bytes = ((size_t)units * n_chunks * d->D * sizeof(float) + 255) / 256 * 256;
-  pl->total_bytes = pl->acc_bytes + ((size_t)units * n_chunks * sizeof(float2) + 255) / 256 * 256;
+  pl->acc_bytes = ((size_t)out_units * n_chunks * d->D * sizeof(float) + 255) / 256 * 256;
+  pl->total_bytes = pl->acc_bytes + ((size_t)out_units * n_chunks * sizeof(float2) + 255) / 256 * 256;
   return true;
 }
 
@@ -423,7 +437,15 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   take_kernel_events(&ev_b, &ev_e);
   dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
   void (*kernel)(const DecodeParams);
-  if (mode == kIndex)
+  const bool share = D == 128 && p.kv_group >= 2 && p.kv_group <= kGqaHeads && mode != kBlockMask;
+  if (share) {
+    grid.y = (unsigned)(p.H / p.kv_group);              // one block per K/V head
+    const bool hi = p.kv_group > 8;
+    if (mode == kIndex)
+      kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true> : decode_partial_gqa_kernel<T, kIndex, false>;
+    else
+      kernel = hi ? decode_partial_gqa_kernel<T, kDense, true> : decode_partial_gqa_kernel<T, kDense, false>;
+  } else if (mode == kIndex)
     kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true> : decode_partial_kernel<T, D, kIndex, false>;
   else if (mode == kBlockMask)
     kernel = aligned32 ? decode_partial_kernel<T, D, kBlockMask, true> : decode_partial_kernel<T, D, kBlockMask, false>;

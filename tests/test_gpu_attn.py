@@ -7,7 +7,7 @@ from oracle import ssa_oracle as O
 from paper_2404_09336_b200 import inputs, ssa
 from paper_2404_09336_b200.runner import DecodeStep
 
-from gpu_util import Problem
+from gpu_util import Problem, random_bits
 from parity import assert_parity
 
 pytestmark = pytest.mark.gpu
@@ -287,29 +287,84 @@ def test_strided_views_and_launch_counter():
     assert_parity(out, ref, False, "strided q")
 
 
-def test_grouped_query_heads_share_a_kv_head():
-    # not in the paper (LLaMA-7B is multi-head): H = 8 query heads over H_kv = 2 cache heads
-    B, H, Hkv, T, D = 3, 8, 2, 700, 128
-    p = Problem(B, Hkv, T, D, "bf16", seed=31)               # cache with H_kv heads
-    rng = np.random.default_rng(2)
-    from gpu_util import random_bits
-    p.q_bits = random_bits(rng, (B, H, D), "bf16")
+@pytest.mark.parametrize("H,Hkv,D,dtype", [(8, 2, 128, "bf16"), (8, 4, 128, "f16"), (16, 2, 128, "bf16"),
+                                           (12, 1, 128, "f16"), (32, 2, 128, "bf16"), (6, 2, 128, "bf16"),
+                                           (40, 2, 128, "bf16"), (8, 2, 64, "bf16")])
+def test_grouped_query_heads_share_a_kv_head(H, Hkv, D, dtype):
+    # not in the paper (LLaMA-7B is multi-head): H query heads over H_kv cache heads.  Groups of 2..16 heads with
+    # D = 128 run on the kernel that reads a row once per group (2, 3, 6, 8, 12, 16 heads here); larger groups
+    # and D = 64 on the one-head-per-block kernel.  Poisoned unselected rows, ragged and empty lists, bad entries.
+    B, T = 4, 700
+    p = Problem(B, Hkv, T, D, dtype, seed=31 + H)              # cache with H_kv heads
+    rng = np.random.default_rng(H)
+    p.q_bits = random_bits(rng, (B, H, D), dtype)
     p.H = H
-    p.upload()
-    ctx = [700, 333, 64]
-    counts = [300, 120, 64]
+    ctx = [700, 333, 64, 500]
+    counts = [300, 120, 64, 0]
     index = np.full((B, 704), -1, np.int32)
     for b in range(B):
         index[b, :counts[b]] = np.sort(rng.choice(ctx[b], counts[b], replace=False))
-    out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=700)
-    k_rep, v_rep = np.repeat(p.k_bits, H // Hkv, axis=1), np.repeat(p.v_bits, H // Hkv, axis=1)
-    ref, ref_lse = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, index, counts, scale_of(D), "bf16")
-    assert status == 0
-    assert_parity(out, ref, False, "grouped queries")
-    np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
-    out_d, _, _ = p.dense(ctx)
-    ref_d, _ = O.decode_attn_dense(p.q_bits, k_rep, v_rep, ctx, scale_of(D), "bf16")
+    nan = 0x7FC0 if dtype == "bf16" else 0x7E00
+    for b in range(B):                                         # rows nobody selects hold NaN
+        unselected = np.setdiff1d(np.arange(T), index[b, :counts[b]])
+        p.k_bits[b][:, unselected] = nan
+        p.v_bits[b][:, unselected] = nan
+    p.upload()
+    g = H // Hkv
+    k_rep, v_rep = np.repeat(p.k_bits, g, axis=1), np.repeat(p.v_bits, g, axis=1)
+    for ms in (700, 300):                                      # several chunks per request / one
+        out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=ms)
+        ref, ref_lse = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, index, counts, scale_of(D), dtype)
+        assert status == 0
+        assert not out[3].any() and np.all(np.isneginf(lse[3]))
+        assert_parity(out, ref, False, f"grouped queries ms={ms}")
+        np.testing.assert_allclose(lse[:3], ref_lse[:3], rtol=1e-5, atol=1e-5)
+    out, _, _, _ = p.sparse(ctx, index, counts, max_selected=700, out_dtype=None)
+    assert_parity(out, ref, True, "grouped queries, output in the storage type")
+    # an entry outside the context is skipped and flagged
+    bad = index.copy()
+    bad[0, 5], bad[1, 0] = 700, -3
+    out, lse, status, _ = p.sparse(ctx, bad, counts, max_selected=700)
+    keep = [np.delete(bad[0, :300], 5), bad[1, 1:120], bad[2, :64], bad[3, :0]]
+    want = np.full((B, 704), -1, np.int32)
+    for b in range(B):
+        want[b, :len(keep[b])] = keep[b]
+    ref_b, _ = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, want, [len(x) for x in keep], scale_of(D), dtype)
+    assert status == ssa.DEV_BAD_INDEX
+    assert_parity(out, ref_b, False, "grouped queries, bad entries")
+    # full context (clean cache)
+    q = Problem(B, Hkv, T, D, dtype, seed=77 + H)
+    q.q_bits = random_bits(rng, (B, H, D), dtype)
+    q.H = H
+    q.upload()
+    out_d, lse_d, _ = q.dense(ctx)
+    ref_d, ref_lse_d = O.decode_attn_dense(q.q_bits, np.repeat(q.k_bits, g, axis=1), np.repeat(q.v_bits, g, axis=1),
+                                           ctx, scale_of(D), dtype)
     assert_parity(out_d, ref_d, False, "grouped queries, dense")
+    np.testing.assert_allclose(lse_d, ref_lse_d, rtol=1e-5, atol=1e-5)
+
+
+def test_grouped_query_heads_large_ragged_batch():
+    # every tile shape of the row-sharing kernel: list lengths 0..600 over 300 requests, 8 heads on 2
+    B, H, Hkv, T, D = 300, 8, 2, 600, 128
+    p = Problem(B, Hkv, T, D, "bf16", seed=5)
+    rng = np.random.default_rng(6)
+    p.q_bits = random_bits(rng, (B, H, D), "bf16")
+    p.H = H
+    p.upload()
+    ctx = rng.integers(1, T + 1, size=B).tolist()
+    counts = [int(rng.integers(0, n + 1)) for n in ctx]
+    index = np.full((B, 608), -1, np.int32)
+    for b in range(B):
+        index[b, :counts[b]] = rng.permutation(ctx[b])[:counts[b]]        # unsorted lists
+    out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=600)
+    ref, ref_lse = O.decode_attn_sparse(p.q_bits, np.repeat(p.k_bits, 4, axis=1), np.repeat(p.v_bits, 4, axis=1),
+                                        ctx, index, counts, scale_of(D), "bf16")
+    assert status == 0
+    assert_parity(out, ref, False, "grouped queries, ragged batch")
+    ok = np.isfinite(ref_lse)
+    np.testing.assert_allclose(lse[ok], ref_lse[ok], rtol=1e-5, atol=1e-5)
+    assert np.all(np.isneginf(lse[~ok]))
 
 
 def test_mixed_batch_of_full_context_and_restricted_requests():
