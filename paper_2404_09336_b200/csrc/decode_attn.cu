@@ -442,9 +442,15 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
     grid.y = (unsigned)(p.H / p.kv_group);              // one block per K/V head
     const bool hi = p.kv_group > 8;
     if (mode == kIndex)
-      kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true> : decode_partial_gqa_kernel<T, kIndex, false>;
+      kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kIndex, true, true>
+                               : decode_partial_gqa_kernel<T, kIndex, true, false>)
+                  : (aligned32 ? decode_partial_gqa_kernel<T, kIndex, false, true>
+                               : decode_partial_gqa_kernel<T, kIndex, false, false>);
     else
-      kernel = hi ? decode_partial_gqa_kernel<T, kDense, true> : decode_partial_gqa_kernel<T, kDense, false>;
+      kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kDense, true, true>
+                               : decode_partial_gqa_kernel<T, kDense, true, false>)
+                  : (aligned32 ? decode_partial_gqa_kernel<T, kDense, false, true>
+                               : decode_partial_gqa_kernel<T, kDense, false, false>);
   } else if (mode == kIndex)
     kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true> : decode_partial_kernel<T, D, kIndex, false>;
   else if (mode == kBlockMask)

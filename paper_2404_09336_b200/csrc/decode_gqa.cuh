@@ -74,8 +74,8 @@ constexpr int kGqaHeads = 16;           // M of the mma: most query heads one bl
 constexpr int kGqaPad = 4;              // floats of padding per head row of the block-level combine
 
 // kHi: more than 8 query heads per K/V head (rows 8..15 of the M dimension are live).
-template <typename T, int kMode, bool kHi>
-__global__ void __launch_bounds__(kThreads, 2)
+template <typename T, int kMode, bool kHi, bool kAligned32>
+__global__ void __launch_bounds__(kThreads, kHi ? 2 : 3)
 decode_partial_gqa_kernel(const DecodeParams p) {
   constexpr int D = 128;
   constexpr bool kSparse = kMode != kDense;
@@ -85,6 +85,7 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   __shared__ int32_t s_idx[kSparse ? kMaxChunk : 1];
   __shared__ __align__(16) float s_acc[kWarps][kLiveHeads][D + kGqaPad];
   __shared__ float s_m[kWarps][kLiveHeads], s_l[kWarps][kLiveHeads];
+  __shared__ uint32_t s_q[kHi ? 32 : 16][32];         // query fragments, [word][lane]: the same for every warp
 
   const int chunk_id = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -116,20 +117,23 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       s_idx[i] = v;
     }
   }
-  // query fragments: dims [32j, 32j+32) of heads g and g+8 of this K/V head
-  uint32_t qa[16], qb[16];
-  {
+  // query fragments: dims [32j, 32j+32) of heads g and g+8 of this K/V head.  They are the same for all
+  // warps and live in shared memory: sixteen registers per lane are worth a third block per SM here.
+  if (warp == 0) {
     const T* q0 = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)(kvh * G) * p.q_sh + 32 * j;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint4 a = make_uint4(0u, 0u, 0u, 0u), h8 = make_uint4(0u, 0u, 0u, 0u);
       if (g < G) a = ld_stream_16B(q0 + (int64_t)g * p.q_sh + 8 * i);
       if (kHi && g + 8 < G) h8 = ld_stream_16B(q0 + (int64_t)(g + 8) * p.q_sh + 8 * i);
-      qa[4 * i] = a.x; qa[4 * i + 1] = a.y; qa[4 * i + 2] = a.z; qa[4 * i + 3] = a.w;
-      qb[4 * i] = h8.x; qb[4 * i + 1] = h8.y; qb[4 * i + 2] = h8.z; qb[4 * i + 3] = h8.w;
+      s_q[4 * i][lane] = a.x; s_q[4 * i + 1][lane] = a.y; s_q[4 * i + 2][lane] = a.z; s_q[4 * i + 3][lane] = a.w;
+      if (kHi) {
+        s_q[16 + 4 * i][lane] = h8.x; s_q[16 + 4 * i + 1][lane] = h8.y;
+        s_q[16 + 4 * i + 2][lane] = h8.z; s_q[16 + 4 * i + 3][lane] = h8.w;
+      }
     }
   }
-  if (kSparse) __syncthreads();
+  __syncthreads();
   if (p.dev_status && kvh == 0) {
     const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
     if (f) atomicOr(p.dev_status, f);
@@ -164,9 +168,11 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       if (pos >= 0) {
         const char* src = kbase + (uint64_t)(uint32_t)pos * p.k_row_bytes;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint4 a = ld_stream_16B(src + 16 * i);
-          kf[nt][4 * i] = a.x; kf[nt][4 * i + 1] = a.y; kf[nt][4 * i + 2] = a.z; kf[nt][4 * i + 3] = a.w;
+        for (int i = 0; i < 2; ++i) {                 // whole 32-byte sectors per request
+          Piece pc;
+          load_piece<kAligned32>(pc, src + 32 * i);
+#pragma unroll
+          for (int w = 0; w < 8; ++w) kf[nt][8 * i + w] = pc.w[w];
         }
       } else {
 #pragma unroll
@@ -178,9 +184,10 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       const int pos = row_pos(2 * j + (rr & 1) + 8 * (rr >> 1));
       if (pos >= 0) {
         const char* src = vbase + (uint64_t)(uint32_t)pos * p.v_row_bytes;
-        const uint4 a = ld_stream_16B(src), c4 = ld_stream_16B(src + 16);
-        vf[rr][0] = a.x; vf[rr][1] = a.y; vf[rr][2] = a.z; vf[rr][3] = a.w;
-        vf[rr][4] = c4.x; vf[rr][5] = c4.y; vf[rr][6] = c4.z; vf[rr][7] = c4.w;
+        Piece pc;
+        load_piece<kAligned32>(pc, src);
+#pragma unroll
+        for (int w = 0; w < 8; ++w) vf[rr][w] = pc.w[w];
       } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) vf[rr][i] = 0u;          // weight 0 times anything stored there must stay 0
@@ -194,8 +201,8 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
-        mma_16816<T>(s[nt], qa[2 * ks], qb[2 * ks], qa[2 * ks + 1], qb[2 * ks + 1], kf[nt][2 * ks],
-                     kf[nt][2 * ks + 1], s[nt]);
+        mma_16816<T>(s[nt], s_q[2 * ks][lane], kHi ? s_q[16 + 2 * ks][lane] : 0u, s_q[2 * ks + 1][lane],
+                     kHi ? s_q[16 + 2 * ks + 1][lane] : 0u, kf[nt][2 * ks], kf[nt][2 * ks + 1], s[nt]);
     }
     // lane (g, j) now holds, for heads g (s[.][0..1]) and g+8 (s[.][2..3]), the rows nt*8 + 2j + {0, 1}
     float mt_lo = neg_inf(), mt_hi = neg_inf();
