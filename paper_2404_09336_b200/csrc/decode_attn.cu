@@ -114,9 +114,12 @@ __device__ __forceinline__ void zero_piece(Piece& r) {
   for (int i = 0; i < 8; ++i) r.w[i] = 0u;
 }
 
-template <typename T, int D, int kMode, bool kAligned32>
+// kPaged (index lists only): positions are translated through the page table while they are staged, and a
+// missing list stands for 0, 1, 2, ...; kept out of the unpaged instantiations so that they stay as they are.
+template <typename T, int D, int kMode, bool kAligned32, bool kPaged = false>
 __global__ void __launch_bounds__(kThreads, SSA_MIN_BLOCKS)
 decode_partial_kernel(const DecodeParams p) {
+  static_assert(!kPaged || kMode == kIndex, "a paged cache is read through staged positions");
   constexpr bool kSparse = kMode != kDense;           // positions come from shared memory
   constexpr int kLanesPerRow = D / 16;                // 32-byte pieces per row
   constexpr int kRowsPerLoad = 32 / kLanesPerRow;     // rows one warp-wide load covers
@@ -149,11 +152,12 @@ decode_partial_kernel(const DecodeParams p) {
   };
   int32_t raw[kIdxPerThread];
   if (kMode == kIndex) {
-    const int32_t* row = p.index ? p.index + (int64_t)b * p.index_stride + start : nullptr;   // null: 0, 1, 2, ...
+    const bool listed = !kPaged || p.index != nullptr;
+    const int32_t* row = listed ? p.index + (int64_t)b * p.index_stride + start : nullptr;
 #pragma unroll
     for (int j = 0; j < kIdxPerThread; ++j) {
       const int r = staged_row(lane + 32 * j);
-      raw[j] = (r < p.chunk && start + r < p.max_selected) ? (p.index ? __ldg(row + r) : start + r) : -1;
+      raw[j] = (r < p.chunk && start + r < p.max_selected) ? (listed ? __ldg(row + r) : start + r) : -1;
     }
   }
   Piece qraw;
@@ -208,7 +212,7 @@ decode_partial_kernel(const DecodeParams p) {
         int v = raw[j];
         if (v < 0 || v >= n) {
           v = -1; flags |= SSA_DEV_BAD_INDEX; bad = true;
-        } else if (p.page_table) {                    // logical position -> row of the pool
+        } else if (kPaged) {                          // logical position -> row of the pool
           const int page = __ldg(p.page_table + (int64_t)b * p.page_table_stride + (v >> p.page_shift));
           if ((unsigned)page < (unsigned)p.n_pages) v = (page << p.page_shift) | (v & p.page_mask);
           else { v = -1; flags |= SSA_DEV_BAD_INDEX; bad = true; }
@@ -451,7 +455,10 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
                                : decode_partial_gqa_kernel<T, kDense, true, false>)
                   : (aligned32 ? decode_partial_gqa_kernel<T, kDense, false, true>
                                : decode_partial_gqa_kernel<T, kDense, false, false>);
-  } else if (mode == kIndex)
+  } else if (mode == kIndex && p.page_table)
+    kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true, true>
+                       : decode_partial_kernel<T, D, kIndex, false, true>;
+  else if (mode == kIndex)
     kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true> : decode_partial_kernel<T, D, kIndex, false>;
   else if (mode == kBlockMask)
     kernel = aligned32 ? decode_partial_kernel<T, D, kBlockMask, true> : decode_partial_kernel<T, D, kBlockMask, false>;
