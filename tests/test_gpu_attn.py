@@ -287,6 +287,45 @@ def test_strided_views_and_launch_counter():
     assert_parity(out, ref, False, "strided q")
 
 
+@pytest.mark.parametrize("H,Hkv", [(3, 3), (8, 2)])
+@pytest.mark.parametrize("how", ["base", "row_stride"])
+def test_cache_aligned_to_16_but_not_32_bytes(H, Hkv, how):
+    # the 256-bit row loads need 32-byte alignment; a cache that only has the 16 bytes the interface asks for
+    # (base address, or a row stride of D + 8 elements) takes the path with two 128-bit loads per piece
+    B, T, D = 2, 300, 128
+    p = Problem(B, Hkv, T, D, "bf16", seed=41 + H)
+    rng = np.random.default_rng(H)
+    p.q_bits = random_bits(rng, (B, H, D), "bf16")
+    p.H = H
+    p.upload()
+    def carve(t):
+        if how == "base":
+            flat = torch.zeros(t.numel() + 8, dtype=t.dtype, device=t.device)
+            view = flat[8:].view(t.shape)
+        else:
+            wide = torch.zeros((B, Hkv, T, D + 8), dtype=t.dtype, device=t.device)
+            view = wide[..., :D]
+        view.copy_(t)
+        return view
+    p.k, p.v = carve(p.k), carve(p.v)
+    assert p.k.data_ptr() % 16 == 0 and (p.k.data_ptr() % 32 == 16 or p.k.stride(2) % 16 == 8)
+    ctx = [300, 177]
+    counts = [150, 60]
+    index = np.full((B, 304), -1, np.int32)
+    for b in range(B):
+        index[b, :counts[b]] = np.sort(rng.choice(ctx[b], counts[b], replace=False))
+    g = H // Hkv
+    k_rep, v_rep = np.repeat(p.k_bits, g, axis=1), np.repeat(p.v_bits, g, axis=1)
+    out, lse, status, _ = p.sparse(ctx, index, counts)
+    ref, ref_lse = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, index, counts, scale_of(D), "bf16")
+    assert status == 0
+    assert_parity(out, ref, False, "16-byte aligned cache, sparse")
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+    out_d, _, _ = p.dense(ctx)
+    ref_d, _ = O.decode_attn_dense(p.q_bits, k_rep, v_rep, ctx, scale_of(D), "bf16")
+    assert_parity(out_d, ref_d, False, "16-byte aligned cache, dense")
+
+
 @pytest.mark.parametrize("H,Hkv,D,dtype", [(8, 2, 128, "bf16"), (8, 4, 128, "f16"), (16, 2, 128, "bf16"),
                                            (12, 1, 128, "f16"), (32, 2, 128, "bf16"), (6, 2, 128, "bf16"),
                                            (40, 2, 128, "bf16"), (8, 2, 64, "bf16")])
