@@ -345,8 +345,11 @@ int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, cons
  * this work.  The KV cache is resident state and is never copied.
  *
  * flags = 0: both copies are cudaMemcpyAsync transfers (copy engine).
- * flags = SSA_STEP_COPY_BY_KERNEL: both copies are done by a kernel of the
- * library that reads / writes the host arena across the bus.  For the few
+ * flags = SSA_STEP_COPY_BY_KERNEL: both copies are done by kernels of the
+ * library that read / write the host arena across the bus (when span_offsets,
+ * spans and ctx_lens lie inside the input arena, the copy in is done by extra
+ * blocks of the index kernel, whose other blocks read the span lists from the
+ * host arena meanwhile).  For the few
  * hundred KB that change per decode step this is faster than a copy-engine
  * transfer, whose set-up time dominates at that size.  The host arenas must
  * then be page-locked memory that the device addresses under the same pointer

@@ -2,7 +2,7 @@
 // lists -> span-restricted attention, optional copy out) enqueued by one call.
 #include <algorithm>
 
-#include "ssa_common.cuh"
+#include "fetch_index.cuh"
 
 namespace ssa {
 
@@ -57,17 +57,35 @@ extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s,
   }
   cudaStream_t st = (cudaStream_t)stream;
   int32_t rc;
-  if (s->host_in) {
-    if (by_kernel) {
-      rc = ssa::copy_by_kernel(s->dev_in, s->host_in, s->in_bytes, st);
-      if (rc != SSA_OK) return rc;
-    } else if (cudaMemcpyAsync(s->dev_in, s->host_in, s->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
-      return SSA_ERR_CUDA;
+  // where a pointer into the device arena has its counterpart in the host arena (nullptr: not in the arena)
+  auto host_twin = [&](const void* dev_ptr) -> const int32_t* {
+    const char* d = static_cast<const char*>(dev_ptr);
+    const char* base = static_cast<const char*>(s->dev_in);
+    if (!s->host_in || d < base || d >= base + s->in_bytes) return nullptr;
+    return reinterpret_cast<const int32_t*>(static_cast<const char*>(s->host_in) + (d - base));
+  };
+  const int32_t* h_off = by_kernel ? host_twin(s->span_offsets) : nullptr;
+  const int32_t* h_spans = by_kernel ? host_twin(s->spans) : nullptr;
+  const int32_t* h_ctx = by_kernel ? host_twin(s->ctx_lens) : nullptr;
+  if (h_off && h_spans && h_ctx && desc->B > 0 && desc->B < 60000) {
+    // the span lists are part of what is fetched: expand them straight from the host arena while the same
+    // launch copies the arena in
+    rc = ssa::fetch_and_index(h_off, h_spans, h_ctx, desc->B, s->index, s->index_stride, s->counts, s->dev_status,
+                              s->dev_in, s->host_in, s->in_bytes, st);
+    if (rc != SSA_OK) return rc;
+  } else {
+    if (s->host_in) {
+      if (by_kernel) {
+        rc = ssa::copy_by_kernel(s->dev_in, s->host_in, s->in_bytes, st);
+        if (rc != SSA_OK) return rc;
+      } else if (cudaMemcpyAsync(s->dev_in, s->host_in, s->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        return SSA_ERR_CUDA;
+      }
     }
+    rc = ssa_spans_to_index(s->span_offsets, s->spans, s->ctx_lens, desc->B, s->index, s->index_stride,
+                            s->counts, s->dev_status, stream);
+    if (rc != SSA_OK) return rc;
   }
-  rc = ssa_spans_to_index(s->span_offsets, s->spans, s->ctx_lens, desc->B, s->index, s->index_stride,
-                          s->counts, s->dev_status, stream);
-  if (rc != SSA_OK) return rc;
   rc = ssa_decode_attn_sparse(desc, s->q, s->k_cache, s->v_cache, s->ctx_lens, s->index, s->index_stride,
                               s->counts, s->max_selected, s->out, s->lse, s->workspace, s->workspace_bytes,
                               s->dev_status, stream);

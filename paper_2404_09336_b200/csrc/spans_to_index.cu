@@ -19,6 +19,9 @@
 // resolves the request's references into spans (as ssa_refs_to_spans does) and
 // packs them straight into the keys in shared memory, so the span list never
 // goes through global memory and the step is one launch instead of two.
+#include <algorithm>
+
+#include "fetch_index.cuh"
 #include "refs_resolve.cuh"
 
 namespace ssa {
@@ -35,11 +38,33 @@ struct SpanSource {
   ssa_anchor_tables tables;
 };
 
-template <bool kFromRefs>
+// kFetch: rows of the grid from first_row on do not expand a request but copy n16 16-byte words from page-locked
+// host memory to the device (the step's inputs), while the other rows read their span lists straight from
+// that host memory: the fetch of a decode step's inputs and its index expansion overlap in one launch.
+struct FetchJob {
+  uint4* dst;
+  const uint4* src;
+  size_t n16;
+  int32_t first_row;
+};
+
+template <bool kFromRefs, bool kFetch = false>
 __global__ void __launch_bounds__(kIdxThreads)
 spans_to_index_kernel(const SpanSource src, int32_t* __restrict__ index,
                       int32_t index_stride, int32_t slice, int32_t* __restrict__ counts,
-                      uint32_t* __restrict__ dev_status) {
+                      uint32_t* __restrict__ dev_status, const FetchJob job) {
+  if (kFetch && (int)blockIdx.y >= job.first_row) {
+    grid_dependency_wait();                      // the destination may still be read by the previous kernel
+    const size_t n_threads = (size_t)(gridDim.y - job.first_row) * gridDim.x * kIdxThreads;
+    size_t i = ((size_t)(blockIdx.y - job.first_row) * gridDim.x + blockIdx.x) * kIdxThreads + threadIdx.x;
+    for (; i + n_threads < job.n16; i += 2 * n_threads) {   // two requests in flight per thread
+      const uint4 a = job.src[i], c = job.src[i + n_threads];
+      job.dst[i] = a;
+      job.dst[i + n_threads] = c;
+    }
+    if (i < job.n16) job.dst[i] = job.src[i];
+    return;
+  }
   __shared__ unsigned long long keys[kMaxSpans];
   __shared__ int32_t new_start[kMaxSpans];
   __shared__ int32_t offs[kMaxSpans + 1];
@@ -184,6 +209,34 @@ spans_to_index_kernel(const SpanSource src, int32_t* __restrict__ index,
   }
 }
 
+// ssa_spans_to_index with the span lists read from page-locked host memory (host_* are host addresses the
+// device can use), fused with the copy of `bytes` bytes from src (the same kind of memory) to dst (device).
+int32_t fetch_and_index(const int32_t* host_span_offsets, const int32_t* host_spans, const int32_t* host_ctx_lens,
+                        int32_t B, int32_t* index, int32_t index_stride, int32_t* counts, uint32_t* dev_status,
+                        void* dst, const void* src, size_t bytes, cudaStream_t stream) {
+  if (!host_span_offsets || !host_spans || !host_ctx_lens || !index || !counts || !dst || !src) return SSA_ERR_NULL;
+  if (B <= 0 || index_stride <= 0) return SSA_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(host_spans) % 8 != 0 || bytes % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(dst) % 16 != 0 || reinterpret_cast<uintptr_t>(src) % 16 != 0)
+    return SSA_ERR_ALIGN;
+  int slices = (index_stride + 511) / 512;
+  if (slices > 32) slices = 32;
+  const int32_t slice = (index_stride + slices - 1) / slices;
+  const size_t n16 = bytes / 16;
+  const size_t per_row = (size_t)slices * kIdxThreads * 2;            // two words per thread
+  const int copy_rows = (int)std::min<size_t>((n16 + per_row - 1) / per_row, 148 * 8);
+  if (B + copy_rows > 65535) return SSA_ERR_SHAPE;
+  SpanSource s = {};
+  s.span_offsets = host_span_offsets; s.spans = host_spans; s.ctx_lens = host_ctx_lens;
+  FetchJob job = {reinterpret_cast<uint4*>(dst), reinterpret_cast<const uint4*>(src), n16, B};
+  dim3 grid((unsigned)slices, (unsigned)(B + std::max(copy_rows, 1)));
+  const cudaError_t err = launch_pdl(spans_to_index_kernel<false, true>, grid, dim3(kIdxThreads), stream, s,
+                                     index, index_stride, slice, counts, dev_status, job);
+  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  note_launches(1);
+  return SSA_OK;
+}
+
 }  // namespace ssa
 
 extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t* spans,
@@ -201,7 +254,7 @@ extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t
   src.span_offsets = span_offsets; src.spans = spans; src.ctx_lens = ctx_lens;
   const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel<false>, grid, dim3(ssa::kIdxThreads),
                                           (cudaStream_t)stream, src, index, index_stride, slice, counts,
-                                          dev_status);
+                                          dev_status, ssa::FetchJob{});
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   ssa::note_launches(1);
   return SSA_OK;
@@ -222,7 +275,7 @@ extern "C" int32_t ssa_refs_to_index(const ssa_anchor_tables* tables, int32_t B,
   src.tables = *tables;
   const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel<true>, grid, dim3(ssa::kIdxThreads),
                                           (cudaStream_t)stream, src, index, index_stride, slice, counts,
-                                          dev_status);
+                                          dev_status, ssa::FetchJob{});
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   ssa::note_launches(1);
   return SSA_OK;
