@@ -303,6 +303,10 @@ def measure(torch, ssa, timer, ds, steps, warmup, peak, kernel_pass=True):
         ms = timer.run(lambda i: gs[i % ncopy].replay(), n)
         res[name] = ms / n * 1e3
         del gs
+    # the attention call alone as direct back-to-back launches: programmatic dependent launch hides each
+    # launch's latency behind the previous kernel, so this is the interval between launches, not a duration
+    ms = timer.run(lambda i: (rot(i), ds.attend_sparse()), steps)
+    res["sparse_attn_pipelined_us"] = ms / steps * 1e3
     ds.step()                                   # leave the sparse result in place
     # (d) the main kernel alone: events recorded by the library around it
     if kernel_pass:
@@ -377,6 +381,86 @@ def paper_microbench(torch, ssa, timer, n_iter=20):
                     "ssa_decode_attn_dense (the paper compares with HF attention on an A100: 1.29x overall, "
                     "0.97/1.2/1.6/1.6x at sparsity block 32/64/128/256)",
             "summary": summary, "rows": rows}
+
+
+def variants_outside_the_paper(torch, ssa, timer, n_iter=100):
+    """Grouped query heads and a paged cache, both outside the paper: B = 32 requests, 32 query heads x 128,
+    context 8192, 10 % selected (the cfg 5 recipe), L2-cold by rotating cache copies."""
+    from paper_2404_09336_b200 import inputs
+    from paper_2404_09336_b200.runner import DecodeStep
+    dev = torch.device("cuda", torch.cuda.current_device())
+    B, H, D, T = 32, 32, 128, 8192
+    rows = []
+    for hkv in (8, 4, 2):
+        wl = inputs.make_config(5, density=0.10, B=B, H=hkv)
+        ncopy = max(2, min(8, int(3e9 // (2 * B * hkv * T * D * 2))))
+        ds = DecodeStep(wl, kv_copies=ncopy)
+        q = torch.randn(B, H, D, device=dev).to(ds.q.dtype)
+        out = torch.zeros(B, H, D, dtype=ds.out.dtype, device=dev)
+        lse = torch.zeros(B, H, dtype=torch.float32, device=dev)
+        desc = ssa.make_desc(q, ds.k, ds.v, out, max_ctx=T)
+        ws = torch.empty(max(ssa.decode_workspace_bytes(desc, ds.max_selected), ssa.decode_workspace_bytes(desc, T)),
+                         dtype=torch.uint8, device=dev)
+        ds.build_index()
+        torch.cuda.synchronize()
+        sel = int(ds.counts.sum().item()) * 2 * hkv * D * 2
+
+        def sparse(i):
+            ds.select_copy(i % ncopy)
+            ssa.decode_attn_sparse(desc, q, ds.k, ds.v, ds.ctx_lens, ds.index, ds.counts, ds.max_selected, out, lse,
+                                   ws, ds.status)
+
+        def dense(i):
+            ds.select_copy(i % ncopy)
+            ssa.decode_attn_dense(desc, q, ds.k, ds.v, ds.ctx_lens, out, lse, ws, ds.status)
+
+        for i in range(3):
+            sparse(i), dense(i)
+        ts = timer.run(sparse, n_iter) / n_iter * 1e3
+        td = timer.run(dense, n_iter // 4) / (n_iter // 4) * 1e3
+        rows.append({"H": H, "H_kv": hkv, "sparse_attn_us": round(ts, 2), "dense_us": round(td, 2),
+                     "kv_gbs_sparse": round(sel / ts / 1e3), "kv_gbs_dense": round(B * T * 2 * hkv * D * 2 / td / 1e3)})
+        del ds, ws
+        torch.cuda.empty_cache()
+    # paged cache: cfg 2 shapes, token-major pool, 16-row pages in shuffled order, against the contiguous call
+    wl = inputs.make_config(2)
+    ncopy = 4
+    ds = DecodeStep(wl, kv_copies=ncopy, layout="bthd")
+    ds.build_index()
+    B, H, D, T, ps = wl.B, wl.H, wl.D, wl.max_ctx, 16
+    n_pages = B * T // ps
+    perm = torch.randperm(n_pages, generator=torch.Generator().manual_seed(1)).to(dev)
+    table = perm.to(torch.int32).view(B, T // ps)
+    pools = []
+    for c in range(ncopy):
+        kp = torch.empty((n_pages, ps, H, D), dtype=ds.k_store[c].dtype, device=dev)
+        vp = torch.empty_like(kp)
+        kp[perm] = ds.k_store[c].view(n_pages, ps, H, D)
+        vp[perm] = ds.v_store[c].view(n_pages, ps, H, D)
+        pools.append((kp, vp))
+    desc = ssa.make_desc_paged(ds.q, pools[0][0], pools[0][1], ds.out, max_ctx=T)
+    pg = ssa.make_paging(table, ps, n_pages)
+
+    def paged(i):
+        kp, vp = pools[i % ncopy]
+        ssa.decode_attn_sparse_paged(desc, ds.q, kp, vp, pg, ds.ctx_lens, ds.index, ds.counts, ds.max_selected,
+                                     ds.out, ds.lse, ds.workspace, ds.status)
+
+    def contiguous(i):
+        ds.select_copy(i % ncopy)
+        ds.attend_sparse()
+
+    for i in range(3):
+        paged(i), contiguous(i)
+    tp = timer.run(paged, 4 * n_iter) / (4 * n_iter) * 1e3
+    tc = timer.run(contiguous, 4 * n_iter) / (4 * n_iter) * 1e3
+    del ds, pools
+    torch.cuda.empty_cache()
+    return {"what": "outside the paper: grouped query heads (B=32, 32 query heads x 128, ctx 8192, 10% selected; rows "
+                    "of a K/V head are read once for its whole group) and a paged cache (cfg 2 shapes, 16-row pages "
+                    "in shuffled order, attention call alone)",
+            "grouped_heads": rows,
+            "paged_cfg2": {"page_size": ps, "paged_attn_us": round(tp, 2), "contiguous_attn_us": round(tc, 2)}}
 
 
 def run_ours(args):
@@ -464,6 +548,7 @@ def run_ours(args):
                 "frac_of_spec_8000": (main["selected_bytes"] / kernel_us / 1e3 / SPEC_HBM_GBS) if kernel_us else None,
                 "traffic": traffic, "kernel_us": kernel_us, "kernel_us_how": kernel_note,
                 "kernel_us_events_hook": main.get("kernel_us"),
+                "launch_interval_us_back_to_back": main.get("sparse_attn_pipelined_us"),
                 "algorithmic_bytes_per_launch": main["selected_bytes"]}
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
@@ -479,7 +564,7 @@ def run_ours(args):
         "speedup_vs_dense": main["speedup_vs_dense"], "density": main["density"],
         "us_per_step": ms / steps * 1e3,
         "breakdown_us": {k: main[k] for k in ("direct_us", "graph_us", "index_us", "sparse_attn_us", "dense_us",
-                                              "warm_us")},
+                                              "warm_us", "sparse_attn_pipelined_us")},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "us_per_step": ms_e2e / steps * 1e3, "copies": e2e_how,
@@ -531,6 +616,7 @@ def run_ours(args):
         line["crossover_density"] = cross
         if args.sweep != "none":
             line["paper_microbench"] = paper_microbench(torch, ssa, timer)
+            line["variants"] = variants_outside_the_paper(torch, ssa, timer)
         line["cpu_baseline"] = time_oracle(args.cfg, budget_s=15.0)
         for k in ("seconds", "ms_per_step", "steps"):
             line["cpu_baseline"].pop(k, None)

@@ -548,3 +548,39 @@ def test_side_stream_graph_replay_and_determinism():
     k, v = wl.kv_bits()
     refd, _ = O.decode_attn_dense(wl.q_bits(), k, v, wl.ctx_lens, scale_of(wl.D), wl.dtype)
     assert_parity(ds.out_f64(), refd, False, "dense from a graph")
+
+
+def test_host_driven_step_replayed_from_a_graph_with_new_inputs():
+    # ssa_decode_step with kernel copies captured once; between replays the host rewrites the pinned input
+    # arena (other query rows, other spans) and the cache changes: every replay must pick the new bytes up
+    kw = dict(out_dtype=torch.float32, span_capacity=40, index_stride=256, max_selected=256)
+    steps = {name: DecodeStep(inputs.make_config(2, B=6, H=4, first_id=fid), **kw) for name, fid in (("a", 0), ("b", 50))}
+    want, arena, cache = {}, {}, {}
+    for name, d in steps.items():
+        d.step()
+        torch.cuda.synchronize()
+        want[name] = (d.out.cpu(), d.lse.cpu(), d.counts.cpu())
+        arena[name] = d.in_arena.cpu()
+        cache[name] = (d.k.clone(), d.v.clone())
+    assert not torch.equal(want["a"][0], want["b"][0]) and arena["a"].shape == arena["b"].shape
+    ds = steps["a"]
+    ds.make_host_buffers()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    ds.step_from_host(direct=True, stream=side)                # first call outside the capture
+    side.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        ds.step_from_host(direct=True)
+    for name in ("a", "b", "a"):
+        ds.h_in.copy_(arena[name])
+        ds.k.copy_(cache[name][0])
+        ds.v.copy_(cache[name][1])
+        ds.h_out.fill_(9)
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        out, lse, counts = want[name]
+        assert torch.equal(ds.h_counts, counts), name
+        assert torch.equal(ds.h_out_rows, out) and torch.equal(ds.h_lse, lse), name
+        assert int(ds.h_status.item()) == 0
