@@ -129,6 +129,29 @@ def test_attention_from_blocked_lists(bs, dtype, D):
     np.testing.assert_allclose(out, out_i, rtol=0, atol=2e-6)
 
 
+def test_blocked_lists_with_grouped_query_heads():
+    # 8 query heads on 2 cache heads through the blocked lists (served by the one-head-per-block kernel)
+    from gpu_util import random_bits
+    B, H, Hkv, T, D, bs = 3, 8, 2, 1000, 128, 64
+    p = Problem(B, Hkv, T, D, "bf16", seed=9)
+    p.q_bits = random_bits(np.random.default_rng(1), (B, H, D), "bf16")
+    p.H = H
+    p.upload()
+    ctx = [1000, 400, 77]
+    lists = [[(0, 64), (300, 420), (900, 1000)], [(10, 390)], [(0, 77)]]
+    offs = np.zeros(B + 1, np.int64)
+    offs[1:] = np.cumsum([len(s) for s in lists])
+    flat = [q for s in lists for q in s]
+    stride = (T + bs - 1) // bs
+    r_idx, r_mask, r_cnt, _ = O.spans_to_blockmask_batch(offs, flat, ctx, bs, stride)
+    k_rep, v_rep = np.repeat(p.k_bits, H // Hkv, axis=1), np.repeat(p.v_bits, H // Hkv, axis=1)
+    ref, ref_lse = O.decode_attn_blockmask(p.q_bits, k_rep, v_rep, ctx, r_idx, r_mask, r_cnt, bs, 1 / np.sqrt(D), "bf16")
+    out, lse, status = attention_from_lists(p, ctx, r_idx, r_mask, r_cnt, bs, stride)
+    assert status == 0
+    assert_parity(out, ref, False, "blocked lists, grouped heads")
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+
+
 def test_end_to_end_on_device_and_bad_bits():
     # spans -> blocked lists -> attention without leaving the device
     wl = inputs.make_config(2, B=5, H=4)

@@ -72,7 +72,8 @@ def random_lists(rng, ctx, stride):
 
 
 @pytest.mark.parametrize("page_size", [1, 16, 128])
-@pytest.mark.parametrize("B,H,H_kv,D,dtype", [(3, 4, 4, 128, "bf16"), (40, 4, 2, 64, "f16")])
+@pytest.mark.parametrize("B,H,H_kv,D,dtype", [(3, 4, 4, 128, "bf16"), (40, 4, 2, 64, "f16"), (5, 8, 2, 128, "bf16"),
+                                              (3, 12, 1, 128, "f16")])
 def test_sparse_and_dense_over_shuffled_pages(page_size, B, H, H_kv, D, dtype):
     T = 700
     p = PagedProblem(B, H, H_kv, D, T, page_size, spare_pages=5, dtype=dtype, seed=page_size + B)
