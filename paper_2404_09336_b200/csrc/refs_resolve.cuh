@@ -43,12 +43,20 @@ __device__ __forceinline__ int resolve_refs_warp(const ssa_anchor_tables& t, int
         flags |= SSA_DEV_BAD_REF;
       }
     }
-    // anchors that do not resolve are dropped, so count what each lane really emits
+    // anchors that do not resolve are dropped, so count what each lane really emits (table reads four at a
+    // time: a lane's walk over its anchors is a chain of dependent-looking loads otherwise)
     int emit = 0;
     if (by_anchor) {
-      for (int a = first; a < first + count; ++a) {
-        const int li = a < n_anchors ? t.anchor_line[a0 + a] : -1;
-        if (li >= 0 && li < n_lines) ++emit; else flags |= SSA_DEV_BAD_REF;
+      for (int a = first; a < first + count; a += 4) {
+        int li[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          li[k] = (a + k < first + count && a + k < n_anchors) ? __ldg(t.anchor_line + a0 + a + k) : -1;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (a + k >= first + count) break;
+          if (li[k] >= 0 && li[k] < n_lines) ++emit; else flags |= SSA_DEV_BAD_REF;
+        }
       }
     } else {
       emit = count;
@@ -61,9 +69,18 @@ __device__ __forceinline__ int resolve_refs_warp(const ssa_anchor_tables& t, int
     }
     int at = written + incl - emit;
     if (by_anchor) {
-      for (int a = first; a < first + count; ++a) {
-        const int li = a < n_anchors ? t.anchor_line[a0 + a] : -1;
-        if (li >= 0 && li < n_lines) put(at++, lines[li]);
+      for (int a = first; a < first + count; a += 4) {
+        int li[4];
+        int2 span[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          li[k] = (a + k < first + count && a + k < n_anchors) ? __ldg(t.anchor_line + a0 + a + k) : -1;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          span[k] = (li[k] >= 0 && li[k] < n_lines) ? __ldg(lines + li[k]) : make_int2(0, 0);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (li[k] >= 0 && li[k] < n_lines) put(at++, span[k]);
       }
     } else if (count == 1) {
       put(at, lines[first]);
