@@ -21,6 +21,8 @@
 // position (dense), a slice of the request's index list, or a run of entries
 // of the request's blocked (block index, bitmask) list, whose set bits the
 // block expands into positions in shared memory before reading any row.
+#include <algorithm>
+
 #include "ssa_common.cuh"
 
 namespace ssa {
@@ -395,6 +397,15 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   int chunk = 256;
   if (max_selected <= kMaxChunk && (units >= 148 || max_selected <= 256)) chunk = kMaxChunk;
   else while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
+  if (shares_rows(d) && max_selected > kMaxChunk) {
+    // The row-sharing kernel leaves G triples per chunk and its blocks are long: fewer, larger chunks
+    // (its blocks walk a chunk in windows of the staging area).  About 2048 blocks for groups of up to 8
+    // heads, one block per resident slot for larger groups (measured, B*H_kv = 64..256, context 8192).
+    const long long target = d->H / d->H_kv > 8 ? 148 * 2 : 2048;
+    long long n = target / units;                              // rounded down: never one block over a full wave
+    n = std::max<long long>(1, std::min<long long>(n, (max_selected + 255) / 256));
+    chunk = std::max(chunk, (int)(((max_selected + n - 1) / n + 63) / 64 * 64));
+  }
   int n_chunks = (max_selected + chunk - 1) / chunk;
   if (n_chunks == 1) chunk = (max_selected + 31) / 32 * 32;
   pl->chunk = chunk;

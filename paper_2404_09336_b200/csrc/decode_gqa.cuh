@@ -102,11 +102,12 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   if (start >= c && chunk_id > 0) return;
   const int cnt = max(0, min(p.chunk, c - start));
 
-  // the block's list entries: checked, translated (paged cache), staged
-  if (kSparse) {
-    const int32_t* row = p.index ? p.index + (int64_t)b * p.index_stride + start : nullptr;
-    for (int i = tid; i < cnt; i += kThreads) {
-      int v = row ? __ldg(row + i) : start + i;
+  // A block may own more list entries than the staging area holds: it works through them in windows of
+  // kMaxChunk entries (checked, translated for a paged cache, staged, consumed).
+  auto stage_window = [&](int w0, int wn) {
+    const int32_t* row = p.index ? p.index + (int64_t)b * p.index_stride + start + w0 : nullptr;
+    for (int i = tid; i < wn; i += kThreads) {
+      int v = row ? __ldg(row + i) : start + w0 + i;
       if (v < 0 || v >= n) {
         v = -1; flags |= SSA_DEV_BAD_INDEX;
       } else if (p.page_table) {
@@ -116,7 +117,8 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       }
       s_idx[i] = v;
     }
-  }
+  };
+  if (kSparse) stage_window(0, min(cnt, kMaxChunk));
   // query fragments: dims [32j, 32j+32) of heads g and g+8 of this K/V head.  They are the same for all
   // warps and live in shared memory: sixteen registers per lane are worth a third block per SM here.
   if (warp == 0) {
@@ -134,11 +136,6 @@ decode_partial_gqa_kernel(const DecodeParams p) {
     }
   }
   __syncthreads();
-  if (p.dev_status && kvh == 0) {
-    const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
-    if (f) atomicOr(p.dev_status, f);
-  }
-
   const char* kbase = reinterpret_cast<const char*>(
       reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)kvh * p.k_sh + 32 * j);
   const char* vbase = reinterpret_cast<const char*>(
@@ -150,12 +147,19 @@ decode_partial_gqa_kernel(const DecodeParams p) {
 #pragma unroll
   for (int u = 0; u < 16; ++u) { o[u][0] = 0.f; o[u][1] = 0.f; o[u][2] = 0.f; o[u][3] = 0.f; }
 
-  for (int t = warp * kGqaRows; t < cnt; t += kWarps * kGqaRows) {
+  for (int w0 = 0; w0 < cnt; w0 += kMaxChunk) {
+  const int wn = min(kMaxChunk, cnt - w0);
+  if (kSparse && w0 > 0) {
+    __syncthreads();                                   // every warp is done with the previous window
+    stage_window(w0, wn);
+    __syncthreads();
+  }
+  for (int t = warp * kGqaRows; t < wn; t += kWarps * kGqaRows) {
     // which of the tile's 16 rows exist (lane r and r+16 both answer for row r)
     int my_pos = -1;
     {
       const int r = t + (lane & 15);
-      if (r < cnt) my_pos = kSparse ? s_idx[r] : start + r;
+      if (r < wn) my_pos = kSparse ? s_idx[r] : start + w0 + r;
     }
     const uint32_t live = __ballot_sync(0xffffffffu, my_pos >= 0) & 0xffffu;
     auto row_pos = [&](int r) { return __shfl_sync(0xffffffffu, my_pos, r); };
@@ -276,6 +280,12 @@ decode_partial_gqa_kernel(const DecodeParams p) {
         o[u][1] = acc[1];
       }
     }
+  }
+
+  }                                                    // windows
+  if (p.dev_status && kvh == 0) {
+    const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
+    if (f) atomicOr(p.dev_status, f);
   }
 
   if (!p.early_release) grid_launch_dependents();
