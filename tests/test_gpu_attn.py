@@ -406,6 +406,47 @@ def test_grouped_query_heads_large_ragged_batch():
     assert np.all(np.isneginf(lse[~ok]))
 
 
+@pytest.mark.parametrize("B,H,Hkv,T", [(350, 4, 2, 1100), (80, 32, 2, 1200)])
+def test_grouped_heads_chunks_longer_than_the_staging_area(B, H, Hkv, T):
+    # with many (request, K/V head) pairs the row-sharing kernel takes chunks of more than 512 entries and walks
+    # them in windows: lists up to the whole context, a bad entry in a late window, sparse and full-context calls
+    D = 128
+    p = Problem(B, Hkv, T, D, "bf16", seed=B)
+    rng = np.random.default_rng(B + 1)
+    p.q_bits = random_bits(rng, (B, H, D), "bf16")
+    p.H = H
+    p.upload()
+    ctx = rng.integers(T // 2, T + 1, size=B).tolist()
+    ctx[0] = T
+    counts = [int(rng.integers(0, n + 1)) for n in ctx]
+    counts[0], counts[1] = T, 1
+    index = np.full((B, T + 4), -1, np.int32)
+    for b in range(B):
+        index[b, :counts[b]] = np.sort(rng.choice(ctx[b], counts[b], replace=False))
+    g = H // Hkv
+    k_rep, v_rep = np.repeat(p.k_bits, g, axis=1), np.repeat(p.v_bits, g, axis=1)
+    sample = sorted(set([0, 1, 2, B // 2, B - 1] + rng.integers(0, B, size=12).tolist()))
+    out, lse, status, _ = p.sparse(ctx, index, counts, max_selected=T)
+    ref, ref_lse = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, index, counts, scale_of(D), "bf16", seqs=sample)
+    assert status == 0
+    assert_parity(out[sample], ref[sample], False, "long chunks")
+    ok = np.isfinite(ref_lse[sample])
+    np.testing.assert_allclose(lse[sample][ok], ref_lse[sample][ok], rtol=1e-5, atol=1e-5)
+    bad = index.copy()
+    bad[0, T - 3] = T + 9                                       # last window of the longest list
+    out, _, status, _ = p.sparse(ctx, bad, counts, max_selected=T)
+    want = index.copy()
+    want[0, :T - 1] = np.delete(index[0, :T], T - 3)
+    cnt2 = list(counts)
+    cnt2[0] = T - 1
+    ref_b, _ = O.decode_attn_sparse(p.q_bits, k_rep, v_rep, ctx, want, cnt2, scale_of(D), "bf16", seqs=[0])
+    assert status == ssa.DEV_BAD_INDEX
+    assert_parity(out[[0]], ref_b[[0]], False, "long chunks, bad entry")
+    out_d, _, _ = p.dense(ctx)
+    ref_d, _ = O.decode_attn_dense(p.q_bits, k_rep, v_rep, ctx, scale_of(D), "bf16", seqs=sample)
+    assert_parity(out_d[sample], ref_d[sample], False, "long chunks, dense")
+
+
 def test_mixed_batch_of_full_context_and_restricted_requests():
     # requests at a "determine span" step attend to everything, the others to their spans, in one launch
     wl = inputs.make_config(2, B=6, H=4)
