@@ -394,25 +394,18 @@ def variants_outside_the_paper(torch, ssa, timer, n_iter=100):
     for hkv in (8, 4, 2):
         wl = inputs.make_config(5, density=0.10, B=B, H=hkv)
         ncopy = max(2, min(8, int(3e9 // (2 * B * hkv * T * D * 2))))
-        ds = DecodeStep(wl, kv_copies=ncopy)
-        q = torch.randn(B, H, D, device=dev).to(ds.q.dtype)
-        out = torch.zeros(B, H, D, dtype=ds.out.dtype, device=dev)
-        lse = torch.zeros(B, H, dtype=torch.float32, device=dev)
-        desc = ssa.make_desc(q, ds.k, ds.v, out, max_ctx=T)
-        ws = torch.empty(max(ssa.decode_workspace_bytes(desc, ds.max_selected), ssa.decode_workspace_bytes(desc, T)),
-                         dtype=torch.uint8, device=dev)
+        ds = DecodeStep(wl, kv_copies=ncopy, query_heads=H)
         ds.build_index()
         torch.cuda.synchronize()
         sel = int(ds.counts.sum().item()) * 2 * hkv * D * 2
 
         def sparse(i):
             ds.select_copy(i % ncopy)
-            ssa.decode_attn_sparse(desc, q, ds.k, ds.v, ds.ctx_lens, ds.index, ds.counts, ds.max_selected, out, lse,
-                                   ws, ds.status)
+            ds.attend_sparse()
 
         def dense(i):
             ds.select_copy(i % ncopy)
-            ssa.decode_attn_dense(desc, q, ds.k, ds.v, ds.ctx_lens, out, lse, ws, ds.status)
+            ds.attend_dense()
 
         for i in range(3):
             sparse(i), dense(i)
@@ -420,7 +413,7 @@ def variants_outside_the_paper(torch, ssa, timer, n_iter=100):
         td = timer.run(dense, n_iter // 4) / (n_iter // 4) * 1e3
         rows.append({"H": H, "H_kv": hkv, "sparse_attn_us": round(ts, 2), "dense_us": round(td, 2),
                      "kv_gbs_sparse": round(sel / ts / 1e3), "kv_gbs_dense": round(B * T * 2 * hkv * D * 2 / td / 1e3)})
-        del ds, ws
+        del ds
         torch.cuda.empty_cache()
     # paged cache: cfg 2 shapes, token-major pool, 16-row pages in shuffled order, against the contiguous call
     wl = inputs.make_config(2)

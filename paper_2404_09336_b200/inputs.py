@@ -87,11 +87,13 @@ class Workload:
             self.seq_ids = np.arange(self.B, dtype=np.int64)
 
     # ---- inputs ------------------------------------------------------------
-    def q_bits(self) -> np.ndarray:
-        """uint16 [B, H, D]."""
-        out = np.empty((self.B, self.H, self.D), np.uint16)
+    def q_bits(self, heads: int | None = None) -> np.ndarray:
+        """uint16 [B, heads, D]; ``heads`` defaults to H (more query heads than
+        cache heads: grouped query heads, which the paper's model does not have)."""
+        heads = heads or self.H
+        out = np.empty((self.B, heads, self.D), np.uint16)
         for i, b in enumerate(self.seq_ids):
-            out[i] = _normal_bits(_rng(self.seed, b, 2), (self.H, self.D), self.dtype)
+            out[i] = _normal_bits(_rng(self.seed, b, 2), (heads, self.D), self.dtype)
         return out
 
     def kv_bits_seq(self, i: int):

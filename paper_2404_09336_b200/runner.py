@@ -55,12 +55,14 @@ class DecodeStep:
     layout "bthd": cache stored [B, T, H, D] (token-major).  Either way
     ``self.k`` / ``self.v`` are the logical [B, H, T, D] views.
     ``kv_copies`` > 1 keeps several copies of the cache so that consecutive
-    timed steps read different memory.
+    timed steps read different memory.  ``query_heads`` (a multiple of the
+    workload's H) gives the query, output and lse that many heads over the
+    workload's H cache heads (grouped query heads).
     """
 
     def __init__(self, wl: Workload, device="cuda:0", layout="bhtd", out_dtype=None, kv_copies=1,
                  index_stride=None, max_selected=None, gen_threads=None,
-                 span_capacity=0):
+                 span_capacity=0, query_heads=None):
         self.wl, self.device, self.layout = wl, torch.device(device), layout
         dt = _TORCH_DTYPE[wl.dtype]
         dev = self.device
@@ -91,13 +93,16 @@ class DecodeStep:
         self.max_selected = int(max_selected or max(wl.selected_upper_bound(), 1))
         self.index_stride = int(index_stride or (self.max_selected + 31) // 32 * 32)
         odt = out_dtype or dt
+        QH = int(query_heads or H)
+        if QH % H != 0:
+            raise ValueError("query_heads must be a multiple of the workload's heads")
         # what changes every decode step lives in one input arena and one result
         # arena, so that a host-driven step is one copy in and one copy out
         self.in_arena, (self.q, self.ctx_lens, self.span_offsets, self.spans) = _arena(
-            dev, [((B, H, D), dt), ((B,), torch.int32), ((B + 1,), torch.int32), ((max(len(spans), span_capacity), 2), torch.int32)])
-        self._out_specs = [((B, H, D), odt), ((B, H), torch.float32), ((B,), torch.int32), ((1,), torch.int32)]
+            dev, [((B, QH, D), dt), ((B,), torch.int32), ((B + 1,), torch.int32), ((max(len(spans), span_capacity), 2), torch.int32)])
+        self._out_specs = [((B, QH, D), odt), ((B, QH), torch.float32), ((B,), torch.int32), ((1,), torch.int32)]
         self.out_arena, (self.out, self.lse, self.counts, self.status) = _arena(dev, self._out_specs)
-        self.q.copy_(bits_to_tensor(wl.q_bits(), wl.dtype))
+        self.q.copy_(bits_to_tensor(wl.q_bits(QH), wl.dtype))
         self.ctx_lens.copy_(torch.from_numpy(wl.ctx_lens.copy()))
         self.span_offsets.copy_(torch.from_numpy(wl.span_offsets.copy()))
         self.spans[: len(spans)].copy_(torch.from_numpy(np.ascontiguousarray(spans)))

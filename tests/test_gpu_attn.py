@@ -625,3 +625,23 @@ def test_host_driven_step_replayed_from_a_graph_with_new_inputs():
         assert torch.equal(ds.h_counts, counts), name
         assert torch.equal(ds.h_out_rows, out) and torch.equal(ds.h_lse, lse), name
         assert int(ds.h_status.item()) == 0
+
+
+def test_decode_step_with_more_query_heads_than_cache_heads():
+    # the runner's buffers with grouped query heads: span lists -> index lists -> attention, 8 query heads on 2
+    wl = inputs.make_config(3, B=2, H=2)
+    ds = DecodeStep(wl, out_dtype=torch.float32, query_heads=8)
+    ds.step()
+    torch.cuda.synchronize()
+    assert int(ds.status.item()) == 0
+    k, v = wl.kv_bits()
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, ds.index_stride)
+    ref, ref_lse = O.decode_attn_sparse(wl.q_bits(8), np.repeat(k, 4, axis=1), np.repeat(v, 4, axis=1), wl.ctx_lens,
+                                        index, counts, scale_of(wl.D), wl.dtype)
+    assert_parity(ds.out_f64(), ref, False, "runner, grouped heads")
+    np.testing.assert_allclose(ds.lse.double().cpu().numpy(), ref_lse, rtol=1e-5, atol=1e-5)
+    ds.attend_dense()
+    torch.cuda.synchronize()
+    refd, _ = O.decode_attn_dense(wl.q_bits(8), np.repeat(k, 4, axis=1), np.repeat(v, 4, axis=1), wl.ctx_lens,
+                                  scale_of(wl.D), wl.dtype)
+    assert_parity(ds.out_f64(), refd, False, "runner, grouped heads, dense")
