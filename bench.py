@@ -542,6 +542,8 @@ def run_ours(args):
                 "traffic": traffic, "kernel_us": kernel_us, "kernel_us_how": kernel_note,
                 "kernel_us_events_hook": main.get("kernel_us"),
                 "launch_interval_us_back_to_back": main.get("sparse_attn_pipelined_us"),
+                "frac_at_launch_interval": (main["selected_bytes"] / main["sparse_attn_pipelined_us"] / 1e3 / peak
+                                            if main.get("sparse_attn_pipelined_us") else None),
                 "algorithmic_bytes_per_launch": main["selected_bytes"]}
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
