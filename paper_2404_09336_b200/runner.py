@@ -143,6 +143,7 @@ class DecodeStep:
         B, dev = self.wl.B, self.device
         self.block_size = block_size
         self.block_stride = (self.wl.max_ctx + block_size - 1) // block_size
+        self._bound_blocks()
         self.block_idx = torch.full((B, self.block_stride), -7, dtype=torch.int32, device=dev)
         self.block_mask = torch.zeros((B, self.block_stride, block_size // 32), dtype=torch.int32, device=dev)
         self.block_counts = torch.zeros((B,), dtype=torch.int32, device=dev)
@@ -150,13 +151,18 @@ class DecodeStep:
         if need > self.workspace.numel():
             self.workspace = torch.empty(need, dtype=torch.uint8, device=dev)
 
+    def _bound_blocks(self):
+        """Host-side bound on the listed blocks of any request: no more than its context spans."""
+        longest = int(self.wl.ctx_lens.max()) if len(self.wl.ctx_lens) else 1
+        self.max_blocks = max(1, min(self.block_stride, (longest + self.block_size - 1) // self.block_size))
+
     def build_blockmask(self, stream=None):
         return ssa.spans_to_blockmask(self.span_offsets, self.spans, self.ctx_lens, self.block_size, self.block_idx,
                                       self.block_mask, self.block_counts, self.status, stream)
 
     def attend_blockmask(self, stream=None):
         return ssa.decode_attn_blockmask(self.desc, self.q, self.k, self.v, self.ctx_lens, self.block_idx,
-                                         self.block_mask, self.block_counts, self.block_size, self.block_stride,
+                                         self.block_mask, self.block_counts, self.block_size, self.max_blocks,
                                          self.out, self.lse, self.workspace, self.status, stream)
 
     def step_blockmask(self, stream=None):
@@ -217,6 +223,8 @@ class DecodeStep:
         self.ctx_lens.copy_(torch.from_numpy(wl.ctx_lens.copy()))
         self.max_selected = max(wl.selected_upper_bound(), 1)
         self.wl = wl
+        if hasattr(self, "block_size"):
+            self._bound_blocks()
 
     # ---- results ---------------------------------------------------------------------
     def out_f64(self) -> np.ndarray:
