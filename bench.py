@@ -141,7 +141,7 @@ def time_oracle(cfg, budget_s, steps=None, warmup=0):
 
     from oracle import ssa_oracle as O
     from paper_2404_09336_b200 import inputs
-    wl = inputs.make_config(cfg)
+    wl = inputs.make_config(cfg, density=0.10 if cfg == 5 else None)
     stride = (wl.selected_upper_bound() + 31) // 32 * 32
     with threadpool_limits(limits=1):
         probe = min(wl.B, 4)
