@@ -4,8 +4,8 @@
 //
 // One thread block per request.  The request's spans are clamped into shared
 // memory once; the context is then swept in windows of kWindowBits positions:
-// every thread owns one 32-bit word of the window's bitmap and ORs in its
-// overlap with each span, the words of a block are tested for emptiness, a
+// the warps OR the spans, one span per warp at a time, into the window's bitmap
+// in shared memory, the words of a block are tested for emptiness, a
 // ballot scan numbers the non-empty blocks of the window after those of the
 // earlier windows, and they are written out.
 #include "ssa_common.cuh"
@@ -49,15 +49,22 @@ spans_to_blockmask_kernel(const int32_t* __restrict__ span_offsets, const int32_
   const int blocks_per_window = kBmThreads / wpb;
   int listed = 0;                                       // non-empty blocks found so far
   for (int w0 = 0; w0 < n; w0 += kWindowBits) {
-    // this thread's word covers positions [lo, lo + 32)
-    const int lo = w0 + tid * 32;
-    uint32_t word = 0;
-    for (int i = 0; i < S; ++i) {
+    // word t of the window's bitmap covers positions [w0 + 32 t, w0 + 32 t + 32).  A warp takes a span at a
+    // time and its lanes OR the span's overlap into the words it touches, so the work follows the total
+    // length of the spans, not spans x words.
+    s_word[tid] = 0u;
+    __syncthreads();
+    for (int i = warp; i < S; i += kBmThreads / 32) {
       const int2 se = s_span[i];
-      const int a = max(se.x, lo), e = min(se.y, lo + 32);
-      if (e > a) word |= (e - a == 32) ? 0xffffffffu : (((1u << (e - a)) - 1u) << (a - lo));
+      const int a = max(se.x, w0), e = min(se.y, w0 + kWindowBits);
+      if (e <= a) continue;                             // warp-uniform
+      const int last = (e - 1 - w0) >> 5;
+      for (int w = ((a - w0) >> 5) + lane; w <= last; w += 32) {
+        const int lo = w0 + w * 32;
+        const int aa = max(a, lo), ee = min(e, lo + 32);
+        atomicOr(&s_word[w], (ee - aa == 32) ? 0xffffffffu : (((1u << (ee - aa)) - 1u) << (aa - lo)));
+      }
     }
-    s_word[tid] = word;
     __syncthreads();
     // thread t < blocks_per_window owns block t of the window
     bool nonempty = false;
