@@ -645,3 +645,46 @@ def test_decode_step_with_more_query_heads_than_cache_heads():
     refd, _ = O.decode_attn_dense(wl.q_bits(8), np.repeat(k, 4, axis=1), np.repeat(v, 4, axis=1), wl.ctx_lens,
                                   scale_of(wl.D), wl.dtype)
     assert_parity(ds.out_f64(), refd, False, "runner, grouped heads, dense")
+
+
+def test_largest_batch_the_grid_allows():
+    # 65535 requests (the launch grid's limit in that dimension), one head, tiny contexts: index expansion,
+    # restricted and full-context attention on sampled requests; one request more is refused on the host
+    B, H, T, D = 65535, 1, 8, 64
+    rng = np.random.default_rng(12)
+    q_bits = random_bits(rng, (B, H, D), "f16")
+    k_bits = random_bits(rng, (B, H, T, D), "f16")
+    v_bits = random_bits(rng, (B, H, T, D), "f16")
+    from paper_2404_09336_b200.runner import bits_to_tensor
+    q, k, v = (bits_to_tensor(x, "f16").to("cuda:0") for x in (q_bits, k_bits, v_bits))
+    ctx = rng.integers(1, T + 1, size=B).astype(np.int32)
+    starts = rng.integers(0, T, size=B)
+    spans = np.stack([starts, np.minimum(starts + rng.integers(1, 5, size=B), T + 2)], axis=1).astype(np.int32)
+    offs = np.arange(B + 1, dtype=np.int32)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to("cuda:0")
+    d_ctx, d_sp, d_off = dev(ctx), dev(spans), dev(offs)
+    index = torch.full((B, 8), -7, dtype=torch.int32, device="cuda:0")
+    counts = torch.full((B,), -7, dtype=torch.int32, device="cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    ssa.spans_to_index(d_off, d_sp, d_ctx, index, counts, status)
+    out = torch.zeros((B, H, D), dtype=torch.float32, device="cuda:0")
+    lse = torch.zeros((B, H), dtype=torch.float32, device="cuda:0")
+    desc = ssa.make_desc(q, k, v, out)
+    ws = torch.empty(max(ssa.decode_workspace_bytes(desc, 8), 16), dtype=torch.uint8, device="cuda:0")
+    ssa.decode_attn_sparse(desc, q, k, v, d_ctx, index, counts, 8, out, lse, ws, status)
+    torch.cuda.synchronize()
+    sample = sorted(set([0, 1, B // 2, B - 2, B - 1] + rng.integers(0, B, size=40).tolist()))
+    want_index, want_counts, want_status = O.spans_to_index_batch(offs, spans, ctx, 8)
+    assert torch.equal(counts.cpu(), torch.from_numpy(want_counts))
+    got_index = index.cpu().numpy()
+    for b in sample:
+        assert got_index[b, :want_counts[b]].tolist() == want_index[b, :want_counts[b]].tolist()
+    assert int(status.item()) == (ssa.DEV_CLIPPED if want_status & O.ST_CLIPPED else 0)
+    ref, _ = O.decode_attn_sparse(q_bits, k_bits, v_bits, ctx, want_index, want_counts, scale_of(D), "f16", seqs=sample)
+    assert_parity(out.double().cpu().numpy()[sample], ref[sample], False, "largest batch, sparse")
+    ssa.decode_attn_dense(desc, q, k, v, d_ctx, out, lse, ws, status)
+    torch.cuda.synchronize()
+    ref_d, _ = O.decode_attn_dense(q_bits, k_bits, v_bits, ctx, scale_of(D), "f16", seqs=sample)
+    assert_parity(out.double().cpu().numpy()[sample], ref_d[sample], False, "largest batch, dense")
+    desc.B = 65536
+    assert ssa.decode_attn_dense(desc, q, k, v, d_ctx, out, lse, ws, status, check=False) == ssa.ERR_SHAPE
