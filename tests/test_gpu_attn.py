@@ -7,7 +7,7 @@ from oracle import ssa_oracle as O
 from paper_2404_09336_b200 import inputs, ssa
 from paper_2404_09336_b200.runner import DecodeStep
 
-from gpu_util import Problem, random_bits
+from gpu_util import Problem, random_bits, run_index
 from parity import assert_parity
 
 pytestmark = pytest.mark.gpu
@@ -688,3 +688,28 @@ def test_largest_batch_the_grid_allows():
     assert_parity(out.double().cpu().numpy()[sample], ref_d[sample], False, "largest batch, dense")
     desc.B = 65536
     assert ssa.decode_attn_dense(desc, q, k, v, d_ctx, out, lse, ws, status, check=False) == ssa.ERR_SHAPE
+
+
+def test_one_long_context_with_hundreds_of_spans():
+    # a single request, 300 000 cached tokens, ~250 spans covering ~45 000 of them: the shared-memory sort of the
+    # index kernel, 32 output slices, hundreds of chunks and the second pass
+    B, H, T, D = 1, 2, 300_000, 64
+    p = Problem(B, H, T, D, "f16", seed=77)
+    rng = np.random.default_rng(5)
+    starts = np.sort(rng.integers(0, T - 400, size=250))
+    spans = [(int(s), int(s + rng.integers(1, 400))) for s in starts]
+    rng.shuffle(spans)
+    stride = 65536
+    index, counts, status, _ = run_index([spans], [T], stride)
+    want = O.spans_to_index(spans, T)
+    assert status == 0 and counts[0] == len(want) and 30_000 < len(want) <= stride
+    assert np.array_equal(index[0, :len(want)], want)
+    out, lse, st, _ = p.sparse([T], index, counts.tolist(), max_selected=stride)
+    ref, ref_lse = O.decode_attn_sparse(p.q_bits, p.k_bits, p.v_bits, [T], index, counts, scale_of(D), "f16")
+    assert st == 0
+    assert_parity(out, ref, False, "long context")
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-5, atol=1e-5)
+    out_d, lse_d, _ = p.dense([T])
+    ref_d, ref_lse_d = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, [T], scale_of(D), "f16")
+    assert_parity(out_d, ref_d, False, "long context, dense")
+    np.testing.assert_allclose(lse_d, ref_lse_d, rtol=1e-5, atol=1e-5)
