@@ -49,7 +49,7 @@ WORKLOAD_TEXT = {
 # DRAM traffic of one launch of the sparse decode kernel at cfg 2 (dram__bytes_read.sum +
 # dram__bytes_write.sum, profiles/decode_partial_kernel_cfg2_ncu_full.md), valid only for the kernel
 # source it was captured from.
-NCU_TRAFFIC = {"source_sha256_16": "ea29397a074320b6", "cfg": 2, "bytes_per_launch": 153149696}
+NCU_TRAFFIC = {"source_sha256_16": "d86eb0cd15b3ce3a", "cfg": 2, "bytes_per_launch": 153018624}
 
 
 def kernel_source_hash():
