@@ -173,6 +173,54 @@ int32_t ssa_decode_attn_sparse(const ssa_attn_desc* desc, const void* q,
                                uint32_t* dev_status, void* stream);
 
 /*
+ * Span-restricted decode attention straight from the span lists: the result of
+ * ssa_spans_to_index followed by ssa_decode_attn_sparse, in one kernel and
+ * without an index list in memory (Sec. "CUDA Kernel Design": the attention
+ * span "might consist of non-contiguous token spans"; Sec. "Self-selected
+ * attention span", Token generation; Algorithm 1 with the span list as the
+ * metadata).  Every thread block sorts and merges its request's spans in
+ * shared memory - the union, exactly as ssa_spans_to_index defines it - and
+ * derives the positions of the rows it reads by arithmetic on the merged runs.
+ *
+ * Same span semantics and status bits as ssa_spans_to_index (unsorted,
+ * overlapping, empty, reversed or out-of-range spans), same result and
+ * options as ssa_decode_attn_sparse.  Two host-side bounds size the launch:
+ *   max_spans     >= the number of spans of any request (a caller knows it: it
+ *                 built the lists).  A request with more keeps its first
+ *                 max_spans spans (SSA_DEV_TOO_MANY_SPANS).  Up to 128 spans
+ *                 per request are merged on chip; with a larger bound (up to
+ *                 SSA_MAX_SPANS_PER_SEQ, beyond which it is treated as that)
+ *                 the call expands the lists with the kernel of
+ *                 ssa_spans_to_index first and attends through them - two
+ *                 launches, same results.
+ *   max_selected  >= the number of positions any request attends to.  A
+ *                 request with more keeps the first max_selected, in
+ *                 ascending order (SSA_DEV_OVERFLOW).
+ * Optional outputs, for callers that also want what ssa_spans_to_index would
+ * have written (the lists are bit-identical to its output):
+ *   index_out   dev int32 [B * index_stride] or NULL; index_stride >=
+ *               max_selected when given; entries past the count untouched
+ *   counts_out  dev int32 [B] or NULL
+ *   span_offsets, spans, ctx_lens  dev, as in ssa_spans_to_index
+ *   workspace   dev, >= ssa_decode_spans_workspace_bytes(desc, max_selected,
+ *               max_spans) bytes, 16-byte aligned, no initialisation needed
+ * A paged cache is not supported by this call.
+ * Errors: those of ssa_decode_attn_sparse; SSA_ERR_CAPACITY also for
+ * max_spans <= 0.
+ */
+size_t ssa_decode_spans_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selected,
+                                        int32_t max_spans);
+int32_t ssa_decode_attn_spans(const ssa_attn_desc* desc, const void* q,
+                              const void* k_cache, const void* v_cache,
+                              const int32_t* ctx_lens, const int32_t* span_offsets,
+                              const int32_t* spans, int32_t max_spans,
+                              int32_t max_selected, void* out, float* lse,
+                              int32_t* index_out, int32_t index_stride,
+                              int32_t* counts_out, void* workspace,
+                              size_t workspace_bytes, uint32_t* dev_status,
+                              void* stream);
+
+/*
  * Full-context decode attention, the baseline the method is compared with
  * (Background equations with M = 0; the paper's "determine attention span"
  * steps attend to all preceding context): as above with the implicit list

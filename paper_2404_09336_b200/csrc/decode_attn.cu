@@ -17,12 +17,17 @@
 // unnormalised triple to the workspace and
 // Pass 2 (decode_merge_kernel) combines the chunks of one (request, head).
 //
-// The attended rows of a block come from one of three sources (kMode): every
-// position (dense), a slice of the request's index list, or a run of entries
+// The attended rows of a block come from one of four sources (kMode): every
+// position (dense), a slice of the request's index list, a run of entries
 // of the request's blocked (block index, bitmask) list, whose set bits the
-// block expands into positions in shared memory before reading any row.
+// block expands into positions in shared memory before reading any row, or
+// the request's span list itself, which the block sorts and merges in shared
+// memory and turns into positions by arithmetic (no index list anywhere).
 #include <algorithm>
+#include <type_traits>
 
+#include "fetch_index.cuh"
+#include "span_merge.cuh"
 #include "ssa_common.cuh"
 
 namespace ssa {
@@ -43,7 +48,7 @@ constexpr int kU = SSA_U;              // 32-byte loads in flight per lane, per 
 constexpr int kMaxChunk = 512;         // index entries staged per block
 constexpr int kIdxPerThread = kMaxChunk / kThreads;
 constexpr int kMaskChunk = 512;        // positions a block expands from bitmasks
-enum { kDense = 0, kIndex = 1, kBlockMask = 2 };
+enum { kDense = 0, kIndex = 1, kBlockMask = 2, kSpans = 3 };
 
 struct DecodeParams {
   const void* q;
@@ -55,6 +60,12 @@ struct DecodeParams {
   const int32_t* block_idx; // blocked list only
   const uint32_t* block_mask;
   int32_t block_size, block_stride;
+  const int32_t* span_offsets;  // span lists only: [B+1]
+  const int2* spans;            //   (start, end) pairs
+  int32_t span_cap;             //   spans taken per request (<= kDirectSpans)
+  int32_t* index_out;           //   optional copy of the positions, [B, index_stride]
+  int32_t* counts_out;          //   optional number of positions per request
+  int32_t* ws_counts;           //   the same for the second pass (when n_chunks > 1)
   void* out;
   float* lse;
   float* ws_acc;            // [B*H*n_chunks, D]
@@ -139,6 +150,7 @@ decode_partial_kernel(const DecodeParams p) {
   __shared__ __align__(16) float s_acc[kGroups][D];
   __shared__ float s_m[kGroups], s_l[kGroups];
   __shared__ int s_wcount[kWarps];
+  __shared__ typename std::conditional<kMode == kSpans, SpanRuns, int>::type s_runs;
 
   const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -178,6 +190,15 @@ decode_partial_kernel(const DecodeParams p) {
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
+  if constexpr (kMode == kSpans) {
+    // the request's spans -> disjoint ascending runs in shared memory (every block of the request repeats this)
+    const int first = __ldg(p.span_offsets + b);
+    const int total = merge_spans_block<kThreads>(s_runs, p.spans + first, __ldg(p.span_offsets + b + 1) - first,
+                                                  p.span_cap, n);
+    c = min(total, p.max_selected);
+    if (total > p.max_selected) flags |= SSA_DEV_OVERFLOW;
+    if (tid == 0) flags |= s_runs.flags;
+  }
   if (start >= c && chunk_id > 0) return;             // chunk 0 always reports
   int cnt = max(0, min(p.chunk, c - start));          // list entries of this block; rows, except for bitmasks
 
@@ -212,6 +233,24 @@ decode_partial_kernel(const DecodeParams p) {
       __syncthreads();
     }
     cnt = rows;
+  }
+  if constexpr (kMode == kSpans) {
+    // positions of this warp's tiles, by arithmetic on the runs; head 0 leaves a copy for callers that want the list
+    int32_t* row = (h == 0 && p.index_out) ? p.index_out + (int64_t)b * p.index_stride + start : nullptr;
+#pragma unroll
+    for (int j = 0; j < kIdxPerThread; ++j) {
+      const int r = staged_row(lane + 32 * j);
+      if (r < cnt) {
+        const int v = span_position(s_runs, start + r);
+        s_idx[r] = v;
+        if (row) row[r] = v;
+      }
+    }
+    __syncwarp();
+    if (chunk_id == 0 && h == 0 && tid == 0) {
+      if (p.counts_out) p.counts_out[b] = c;
+      if (p.ws_counts) p.ws_counts[b] = c;
+    }
   }
   bool any_bad = false;                               // warp-uniform: an entry of this warp's tiles is out of range
   if (kMode == kIndex) {
@@ -470,6 +509,11 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
                                : decode_partial_gqa_kernel<T, kIndex, true, false>)
                   : (aligned32 ? decode_partial_gqa_kernel<T, kIndex, false, true>
                                : decode_partial_gqa_kernel<T, kIndex, false, false>);
+    else if (mode == kSpans)
+      kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kSpans, true, true>
+                               : decode_partial_gqa_kernel<T, kSpans, true, false>)
+                  : (aligned32 ? decode_partial_gqa_kernel<T, kSpans, false, true>
+                               : decode_partial_gqa_kernel<T, kSpans, false, false>);
     else
       kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kDense, true, true>
                                : decode_partial_gqa_kernel<T, kDense, true, false>)
@@ -482,6 +526,8 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
     kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true> : decode_partial_kernel<T, D, kIndex, false>;
   else if (mode == kBlockMask)
     kernel = aligned32 ? decode_partial_kernel<T, D, kBlockMask, true> : decode_partial_kernel<T, D, kBlockMask, false>;
+  else if (mode == kSpans)
+    kernel = aligned32 ? decode_partial_kernel<T, D, kSpans, true> : decode_partial_kernel<T, D, kSpans, false>;
   else
     kernel = aligned32 ? decode_partial_kernel<T, D, kDense, true> : decode_partial_kernel<T, D, kDense, false>;
   if (ev_b) cudaEventRecord(ev_b, st);
@@ -490,7 +536,9 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   int launches = 1;
   if (p.n_chunks > 1) {
-    err = launch_pdl(decode_merge_kernel<T, D>, dim3((unsigned)p.H, (unsigned)B), dim3(D), st, p);
+    DecodeParams pm = p;
+    if (mode == kSpans) pm.counts = p.ws_counts;        // the first pass left the list lengths there
+    err = launch_pdl(decode_merge_kernel<T, D>, dim3((unsigned)p.H, (unsigned)B), dim3(D), st, pm);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
     ++launches;
   }
@@ -501,14 +549,23 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
 // A request's attended set in the blocked encoding (mode kBlockMask).
 struct BlockList { const int32_t* block_idx; const uint32_t* block_mask; int32_t block_size; };
 
+// The span lists themselves (mode kSpans), with the optional copies of what they expand to.
+struct SpanLists { const int32_t* span_offsets; const int32_t* spans; int32_t span_cap; int32_t* index_out;
+                   int32_t* counts_out; };
+
+static size_t counts_bytes(const ssa_attn_desc* d) { return ((size_t)d->B * sizeof(int32_t) + 255) / 256 * 256; }
+
 // mode kDense: index/counts unused.  kIndex: the index list.  kBlockMask: `counts`
 // are the numbers of listed blocks, `index_stride` the list capacity in blocks,
-// `max_selected` the host bound on listed blocks, `bl` the lists.
+// `max_selected` the host bound on listed blocks, `bl` the lists.  kSpans: `sl`
+// the span lists, `index_stride` the pitch of sl->index_out; the workspace then
+// ends with one int32 per request (list lengths for the second pass).
 static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const void* v,
                    const int32_t* ctx_lens, const int32_t* index, int32_t index_stride,
                    const int32_t* counts, int32_t max_selected, void* out, float* lse,
                    void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream, int mode,
-                   const BlockList* bl = nullptr, const ssa_paging* pg = nullptr) {
+                   const BlockList* bl = nullptr, const ssa_paging* pg = nullptr,
+                   const SpanLists* sl = nullptr) {
   // a paged cache is read through the staged-positions path; without a list the positions are 0 .. ctx_len-1
   const bool dense_paged = pg && mode == kDense;
   if (dense_paged) mode = kIndex;
@@ -524,11 +581,19 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
       return SSA_ERR_SHAPE;
   }
   if (mode == kBlockMask && (!bl || !bl->block_idx || !bl->block_mask || !counts)) return SSA_ERR_NULL;
+  if (mode == kSpans) {
+    if (!sl || !sl->span_offsets || !sl->spans) return SSA_ERR_NULL;
+    if (pg) return SSA_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(sl->spans) % 8 != 0) return SSA_ERR_ALIGN;
+  }
   const int32_t rc = check_desc(d);
   if (rc != SSA_OK) return rc;
   if (dense_paged) {
     max_selected = d->max_ctx;
     index_stride = d->max_ctx;
+  } else if (mode == kSpans) {
+    if (max_selected <= 0 || sl->span_cap <= 0 || sl->span_cap > kDirectSpans) return SSA_ERR_CAPACITY;
+    if (sl->index_out && max_selected > index_stride) return SSA_ERR_CAPACITY;
   } else if (mode != kDense) {
     if (index_stride <= 0 || max_selected <= 0 || max_selected > index_stride) return SSA_ERR_CAPACITY;
   } else {
@@ -543,13 +608,19 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   } else if (!make_plan(d, max_selected, &pl)) {
     return SSA_ERR_SHAPE;
   }
-  if (!ws || ws_bytes < pl.total_bytes) return SSA_ERR_WORKSPACE;
+  if (!ws || ws_bytes < pl.total_bytes + (mode == kSpans ? counts_bytes(d) : 0)) return SSA_ERR_WORKSPACE;
 
   DecodeParams p;
+  p.span_offsets = mode == kSpans ? sl->span_offsets : nullptr;
+  p.spans = mode == kSpans ? reinterpret_cast<const int2*>(sl->spans) : nullptr;
+  p.span_cap = mode == kSpans ? sl->span_cap : 0;
+  p.index_out = mode == kSpans ? sl->index_out : nullptr;
+  p.counts_out = mode == kSpans ? sl->counts_out : nullptr;
+  p.ws_counts = mode == kSpans ? reinterpret_cast<int32_t*>(reinterpret_cast<char*>(ws) + pl.total_bytes) : nullptr;
   p.q = q; p.k = k; p.v = v;
   p.ctx_lens = ctx_lens;
   p.index = sparse && !dense_paged ? index : nullptr;
-  p.counts = mode != kDense && !dense_paged ? counts : nullptr;
+  p.counts = mode != kDense && mode != kSpans && !dense_paged ? counts : nullptr;
   p.page_table = pg ? pg->page_table : nullptr;
   p.page_table_stride = pg ? pg->page_table_stride : 0;
   p.n_pages = pg ? pg->n_pages : 0;
@@ -629,6 +700,55 @@ int32_t ssa_decode_attn_sparse_noalloc(const ssa_attn_desc* desc, const void* q,
   if (!scratch) return SSA_ERR_CUDA;
   return ssa::run(desc, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out, lse,
                   scratch, SSA_STATIC_SCRATCH_BYTES, dev_status, stream, ssa::kIndex);
+}
+
+// Layout of the workspace of ssa_decode_attn_spans: the partial results of the split pass, one int32 per
+// request, and - only when the request may have more spans than a block merges in shared memory and the
+// list is expanded by ssa_spans_to_index first - room for the index lists.
+static size_t spans_index_pitch(int32_t max_selected) { return ((size_t)max_selected + 31) / 32 * 32; }
+
+size_t ssa_decode_spans_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selected, int32_t max_spans) {
+  ssa::Plan pl;
+  if (!desc || max_spans <= 0 || ssa::check_desc(desc) != SSA_OK || !ssa::make_plan(desc, max_selected, &pl))
+    return 0;
+  size_t need = pl.total_bytes + ssa::counts_bytes(desc);
+  if (max_spans > ssa::kDirectSpans) need += (size_t)desc->B * spans_index_pitch(max_selected) * sizeof(int32_t);
+  return need;
+}
+
+int32_t ssa_decode_attn_spans(const ssa_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* ctx_lens, const int32_t* span_offsets, const int32_t* spans,
+                              int32_t max_spans, int32_t max_selected, void* out, float* lse, int32_t* index_out,
+                              int32_t index_stride, int32_t* counts_out, void* workspace, size_t workspace_bytes,
+                              uint32_t* dev_status, void* stream) {
+  if (!desc || !span_offsets || !spans) return SSA_ERR_NULL;
+  if (max_spans <= 0) return SSA_ERR_CAPACITY;
+  if (max_spans <= ssa::kDirectSpans) {
+    const ssa::SpanLists sl = {span_offsets, spans, max_spans, index_out, counts_out};
+    return ssa::run(desc, q, k_cache, v_cache, ctx_lens, nullptr, index_stride, nullptr, max_selected, out, lse,
+                    workspace, workspace_bytes, dev_status, stream, ssa::kSpans, nullptr, nullptr, &sl);
+  }
+  // More spans per request than a block merges on chip: expand the lists once (into the caller's buffers
+  // when given, else into the workspace) and attend through them.
+  if (!q || !k_cache || !v_cache || !ctx_lens || !out) return SSA_ERR_NULL;
+  const int32_t rc = ssa::check_desc(desc);
+  if (rc != SSA_OK) return rc;
+  ssa::Plan pl;
+  if (max_selected <= 0 || (index_out && max_selected > index_stride)) return SSA_ERR_CAPACITY;
+  if (!ssa::make_plan(desc, max_selected, &pl)) return SSA_ERR_SHAPE;
+  if (!workspace || workspace_bytes < ssa_decode_spans_workspace_bytes(desc, max_selected, max_spans))
+    return SSA_ERR_WORKSPACE;
+  if (!ssa::aligned16(workspace)) return SSA_ERR_ALIGN;
+  char* ws = static_cast<char*>(workspace);
+  int32_t* counts = counts_out ? counts_out : reinterpret_cast<int32_t*>(ws + pl.total_bytes);
+  int32_t* index = index_out ? index_out : reinterpret_cast<int32_t*>(ws + pl.total_bytes + ssa::counts_bytes(desc));
+  const int32_t pitch = index_out ? index_stride : (int32_t)spans_index_pitch(max_selected);
+  const int32_t cap = max_spans < SSA_MAX_SPANS_PER_SEQ ? max_spans : SSA_MAX_SPANS_PER_SEQ;
+  const int32_t rc2 = ssa::spans_to_index_capped(span_offsets, spans, ctx_lens, desc->B, index, pitch, max_selected,
+                                                 cap, counts, dev_status, (cudaStream_t)stream);
+  if (rc2 != SSA_OK) return rc2;
+  return ssa::run(desc, q, k_cache, v_cache, ctx_lens, index, pitch, counts, max_selected, out, lse, workspace,
+                  pl.total_bytes, dev_status, stream, ssa::kIndex);
 }
 
 size_t ssa_decode_blockmask_workspace_bytes(const ssa_attn_desc* desc, int32_t block_size, int32_t max_blocks) {

@@ -80,12 +80,14 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   constexpr int D = 128;
   constexpr bool kSparse = kMode != kDense;
   constexpr int kLiveHeads = kHi ? 16 : 8;
-  static_assert(kMode == kDense || kMode == kIndex, "blocked lists take the one-head-per-block kernel");
+  static_assert(kMode == kDense || kMode == kIndex || kMode == kSpans,
+                "blocked lists take the one-head-per-block kernel");
 
   __shared__ int32_t s_idx[kSparse ? kMaxChunk : 1];
   __shared__ __align__(16) float s_acc[kWarps][kLiveHeads][D + kGqaPad];
   __shared__ float s_m[kWarps][kLiveHeads], s_l[kWarps][kLiveHeads];
   __shared__ uint32_t s_q[kHi ? 32 : 16][32];         // query fragments, [word][lane]: the same for every warp
+  __shared__ typename std::conditional<kMode == kSpans, SpanRuns, int>::type s_runs;
 
   const int chunk_id = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -99,12 +101,34 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
+  if constexpr (kMode == kSpans) {
+    // the request's spans -> disjoint ascending runs in shared memory
+    const int first = __ldg(p.span_offsets + b);
+    const int total = merge_spans_block<kThreads>(s_runs, p.spans + first, __ldg(p.span_offsets + b + 1) - first,
+                                                  p.span_cap, n);
+    c = min(total, p.max_selected);
+    if (total > p.max_selected) flags |= SSA_DEV_OVERFLOW;
+    if (tid == 0) flags |= s_runs.flags;
+    if (chunk_id == 0 && kvh == 0 && tid == 0) {
+      if (p.counts_out) p.counts_out[b] = c;
+      if (p.ws_counts) p.ws_counts[b] = c;
+    }
+  }
   if (start >= c && chunk_id > 0) return;
   const int cnt = max(0, min(p.chunk, c - start));
 
   // A block may own more list entries than the staging area holds: it works through them in windows of
   // kMaxChunk entries (checked, translated for a paged cache, staged, consumed).
   auto stage_window = [&](int w0, int wn) {
+    if constexpr (kMode == kSpans) {                  // positions by arithmetic on the runs
+      int32_t* out = (kvh == 0 && p.index_out) ? p.index_out + (int64_t)b * p.index_stride + start + w0 : nullptr;
+      for (int i = tid; i < wn; i += kThreads) {
+        const int v = span_position(s_runs, start + w0 + i);
+        s_idx[i] = v;
+        if (out) out[i] = v;
+      }
+      return;
+    }
     const int32_t* row = p.index ? p.index + (int64_t)b * p.index_stride + start + w0 : nullptr;
     for (int i = tid; i < wn; i += kThreads) {
       int v = row ? __ldg(row + i) : start + w0 + i;

@@ -36,8 +36,12 @@ __device__ __forceinline__ int resolve_refs_warp(const ssa_anchor_tables& t, int
         if (n_lines + ref.x >= 0) { first = n_lines + ref.x; count = 1; }
         else flags |= SSA_DEV_BAD_REF;
       } else if (ref.x >= 0 && ref.x <= ref.y) {
+        // anchors past the end of the table do not exist: flag them and walk only the ones that do, so the
+        // work per reference is bounded by the table whatever the pair says
+        int hi = ref.y;
+        if (hi >= n_anchors) { hi = n_anchors - 1; flags |= SSA_DEV_BAD_REF; }
         first = ref.x;
-        count = ref.y - ref.x + 1;
+        count = max(hi - ref.x + 1, 0);
         by_anchor = true;
       } else {
         flags |= SSA_DEV_BAD_REF;

@@ -52,7 +52,10 @@ template <bool kFromRefs, bool kFetch = false>
 __global__ void __launch_bounds__(kIdxThreads)
 spans_to_index_kernel(const SpanSource src, int32_t* __restrict__ index,
                       int32_t index_stride, int32_t slice, int32_t* __restrict__ counts,
-                      uint32_t* __restrict__ dev_status, const FetchJob job) {
+                      uint32_t* __restrict__ dev_status, const FetchJob job,
+                      int32_t capacity, int32_t span_cap) {
+  // index_stride: distance between the rows of `index`; capacity <= index_stride: most positions a list keeps;
+  // span_cap <= kMaxSpans: most spans a request may have
   if (kFetch && (int)blockIdx.y >= job.first_row) {
     grid_dependency_wait();                      // the destination may still be read by the previous kernel
     const size_t n_threads = (size_t)(gridDim.y - job.first_row) * gridDim.x * kIdxThreads;
@@ -106,7 +109,7 @@ spans_to_index_kernel(const SpanSource src, int32_t* __restrict__ index,
     S = span_offsets[b + 1] - first;
   }
   if (S < 0) S = 0;
-  if (S > kMaxSpans) { S = kMaxSpans; flags |= SSA_DEV_TOO_MANY_SPANS; }
+  if (S > span_cap) { S = span_cap; flags |= SSA_DEV_TOO_MANY_SPANS; }
   int P = 32;
   while (P < S) P <<= 1;
   __syncthreads();
@@ -188,11 +191,11 @@ spans_to_index_kernel(const SpanSource src, int32_t* __restrict__ index,
   __syncthreads();
 
   const int total = offs[P];
-  const int c = min(total, index_stride);
+  const int c = min(total, capacity);
   if (blockIdx.x == 0 && tid == 0) {
     counts[b] = c;
     uint32_t f = s_flags;
-    if (total > index_stride) f |= SSA_DEV_OVERFLOW;
+    if (total > capacity) f |= SSA_DEV_OVERFLOW;
     if (f && dev_status) atomicOr(dev_status, f);
   }
 
@@ -231,7 +234,29 @@ int32_t fetch_and_index(const int32_t* host_span_offsets, const int32_t* host_sp
   FetchJob job = {reinterpret_cast<uint4*>(dst), reinterpret_cast<const uint4*>(src), n16, B};
   dim3 grid((unsigned)slices, (unsigned)(B + std::max(copy_rows, 1)));
   const cudaError_t err = launch_pdl(spans_to_index_kernel<false, true>, grid, dim3(kIdxThreads), stream, s,
-                                     index, index_stride, slice, counts, dev_status, job);
+                                     index, index_stride, slice, counts, dev_status, job, index_stride, kMaxSpans);
+  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
+  note_launches(1);
+  return SSA_OK;
+}
+
+// ssa_spans_to_index with two more bounds: a list keeps at most `capacity` <= index_stride positions and a
+// request at most `span_cap` <= SSA_MAX_SPANS_PER_SEQ spans.
+int32_t spans_to_index_capped(const int32_t* span_offsets, const int32_t* spans, const int32_t* ctx_lens, int32_t B,
+                              int32_t* index, int32_t index_stride, int32_t capacity, int32_t span_cap,
+                              int32_t* counts, uint32_t* dev_status, cudaStream_t stream) {
+  if (!span_offsets || !spans || !ctx_lens || !index || !counts) return SSA_ERR_NULL;
+  if (B <= 0 || B > 65535 || index_stride <= 0) return SSA_ERR_SHAPE;
+  if (capacity <= 0 || capacity > index_stride || span_cap <= 0 || span_cap > kMaxSpans) return SSA_ERR_CAPACITY;
+  if (reinterpret_cast<uintptr_t>(spans) % 8 != 0) return SSA_ERR_ALIGN;
+  int slices = (capacity + 511) / 512;               // blocks per request: 512 entries each, at most 32
+  if (slices > 32) slices = 32;
+  const int32_t slice = (capacity + slices - 1) / slices;
+  dim3 grid((unsigned)slices, (unsigned)B);
+  SpanSource src = {};
+  src.span_offsets = span_offsets; src.spans = spans; src.ctx_lens = ctx_lens;
+  const cudaError_t err = launch_pdl(spans_to_index_kernel<false>, grid, dim3(kIdxThreads), stream, src, index,
+                                     index_stride, slice, counts, dev_status, FetchJob{}, capacity, span_cap);
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   note_launches(1);
   return SSA_OK;
@@ -243,21 +268,8 @@ extern "C" int32_t ssa_spans_to_index(const int32_t* span_offsets, const int32_t
                                       const int32_t* ctx_lens, int32_t B, int32_t* index,
                                       int32_t index_stride, int32_t* counts,
                                       uint32_t* dev_status, void* stream) {
-  if (!span_offsets || !spans || !ctx_lens || !index || !counts) return SSA_ERR_NULL;
-  if (B <= 0 || B > 65535 || index_stride <= 0) return SSA_ERR_SHAPE;
-  if (reinterpret_cast<uintptr_t>(spans) % 8 != 0) return SSA_ERR_ALIGN;
-  int slices = (index_stride + 511) / 512;           // blocks per request: 512 entries each, at most 32
-  if (slices > 32) slices = 32;
-  const int32_t slice = (index_stride + slices - 1) / slices;
-  dim3 grid((unsigned)slices, (unsigned)B);
-  ssa::SpanSource src = {};
-  src.span_offsets = span_offsets; src.spans = spans; src.ctx_lens = ctx_lens;
-  const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel<false>, grid, dim3(ssa::kIdxThreads),
-                                          (cudaStream_t)stream, src, index, index_stride, slice, counts,
-                                          dev_status, ssa::FetchJob{});
-  if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
-  ssa::note_launches(1);
-  return SSA_OK;
+  return ssa::spans_to_index_capped(span_offsets, spans, ctx_lens, B, index, index_stride, index_stride,
+                                    ssa::kMaxSpans, counts, dev_status, (cudaStream_t)stream);
 }
 
 extern "C" int32_t ssa_refs_to_index(const ssa_anchor_tables* tables, int32_t B, int32_t* index,
@@ -275,7 +287,7 @@ extern "C" int32_t ssa_refs_to_index(const ssa_anchor_tables* tables, int32_t B,
   src.tables = *tables;
   const cudaError_t err = ssa::launch_pdl(ssa::spans_to_index_kernel<true>, grid, dim3(ssa::kIdxThreads),
                                           (cudaStream_t)stream, src, index, index_stride, slice, counts,
-                                          dev_status, ssa::FetchJob{});
+                                          dev_status, ssa::FetchJob{}, index_stride, ssa::kMaxSpans);
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   ssa::note_launches(1);
   return SSA_OK;

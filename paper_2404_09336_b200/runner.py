@@ -112,8 +112,10 @@ class DecodeStep:
         self.status.zero_()
         self.index = torch.full((B, self.index_stride), -7, dtype=torch.int32, device=dev)
         self.desc = ssa.make_desc(self.q, self.k, self.v, self.out, max_ctx=T)
+        self.max_spans = int(max(1, np.diff(wl.span_offsets).max() if wl.B else 1))
         need = max(ssa.decode_workspace_bytes(self.desc, self.max_selected),
-                   ssa.decode_workspace_bytes(self.desc, T))
+                   ssa.decode_workspace_bytes(self.desc, T),
+                   ssa.decode_spans_workspace_bytes(self.desc, self.index_stride, ssa.MAX_SPANS_PER_SEQ))
         if need == 0:
             raise RuntimeError("ssa_decode_workspace_bytes rejected the descriptor")
         self.workspace = torch.empty(need, dtype=torch.uint8, device=dev)
@@ -132,6 +134,13 @@ class DecodeStep:
         return ssa.decode_attn_sparse(self.desc, self.q, self.k, self.v, self.ctx_lens, self.index,
                                       self.counts, self.max_selected, self.out, self.lse, self.workspace,
                                       self.status, stream)
+
+    def attend_spans(self, stream=None, want_lists=False):
+        """Span lists -> attention output in one call (no index list unless want_lists)."""
+        return ssa.decode_attn_spans(self.desc, self.q, self.k, self.v, self.ctx_lens, self.span_offsets, self.spans,
+                                     self.max_spans, self.max_selected, self.out, self.lse,
+                                     self.index if want_lists else None, self.counts if want_lists else None,
+                                     self.workspace, self.status, stream)
 
     def attend_dense(self, stream=None):
         return ssa.decode_attn_dense(self.desc, self.q, self.k, self.v, self.ctx_lens, self.out, self.lse,
@@ -222,6 +231,7 @@ class DecodeStep:
         self.span_offsets.copy_(torch.from_numpy(wl.span_offsets.copy()))
         self.ctx_lens.copy_(torch.from_numpy(wl.ctx_lens.copy()))
         self.max_selected = max(wl.selected_upper_bound(), 1)
+        self.max_spans = int(max(1, np.diff(wl.span_offsets).max()))
         self.wl = wl
         if hasattr(self, "block_size"):
             self._bound_blocks()

@@ -80,6 +80,11 @@ def _load():
     lib.ssa_decode_attn_sparse.restype = C.c_int32
     lib.ssa_decode_attn_sparse.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, C.c_int32, vp, C.c_int32,
                                            vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_spans_workspace_bytes.restype = C.c_size_t
+    lib.ssa_decode_spans_workspace_bytes.argtypes = [C.POINTER(AttnDesc), C.c_int32, C.c_int32]
+    lib.ssa_decode_attn_spans.restype = C.c_int32
+    lib.ssa_decode_attn_spans.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, C.c_int32, C.c_int32, vp, vp,
+                                          vp, C.c_int32, vp, vp, C.c_size_t, vp, vp]
     lib.ssa_spans_to_blockmask.restype = C.c_int32
     lib.ssa_spans_to_blockmask.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp, vp, C.c_int32, vp, vp, vp]
     lib.ssa_decode_blockmask_workspace_bytes.restype = C.c_size_t
@@ -194,6 +199,24 @@ def decode_attn_sparse(desc, q, k_cache, v_cache, ctx_lens, index, counts, max_s
                                     _ptr(counts), int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace),
                                     ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_sparse", rc, check)
+
+
+DIRECT_SPANS = 128      # spans per request the span-list attention call merges on chip
+
+
+def decode_spans_workspace_bytes(desc: AttnDesc, max_selected: int, max_spans: int) -> int:
+    return int(lib.ssa_decode_spans_workspace_bytes(C.byref(desc), int(max_selected), int(max_spans)))
+
+
+def decode_attn_spans(desc, q, k_cache, v_cache, ctx_lens, span_offsets, spans, max_spans, max_selected, out, lse=None,
+                      index_out=None, counts_out=None, workspace=None, dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_spans: span lists -> attention output in one call; index_out / counts_out optional."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_spans(C.byref(desc), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens),
+                                   _ptr(span_offsets), _ptr(spans), int(max_spans), int(max_selected), _ptr(out),
+                                   _ptr(lse), _ptr(index_out), _row_stride(index_out) if index_out is not None else 0,
+                                   _ptr(counts_out), _ptr(workspace), ws_bytes, _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_spans", rc, check)
 
 
 def spans_to_blockmask(span_offsets, spans, ctx_lens, block_size, block_idx, block_mask, block_counts,

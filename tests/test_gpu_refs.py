@@ -154,6 +154,26 @@ def test_one_launch_paper_examples_and_flags():
     compare_index([dict(many, refs=[(0, 699)])], 2816)
 
 
+def test_references_far_beyond_the_anchor_table_cost_nothing_and_are_flagged():
+    """A pair (lo, hi) with hi in the billions must neither be walked anchor by anchor nor lose its flag.
+    The oracle walks every named anchor, so it is given the same pair cut one anchor past the table: the
+    anchors beyond the table contribute nothing but the flag, and that one anchor already raises it."""
+    arith = dict(lines=[(0, 14), (14, 40), (40, 54), (54, 66)], anchors=[0, 2, 3], prefix=0, start=66, ctx=69)
+    for lo in (0, 1, 3, 5):
+        for hi in (1 << 30, 2 ** 31 - 1):
+            on_device = [dict(arith, refs=[(lo, hi), (-1, -1)])]
+            for_oracle = dict(arith, refs=[(lo, max(lo, 3)), (-1, -1)])
+            so, sp, ctx, status = run_refs(on_device, 8)
+            ref, st = O.resolve_references(for_oracle["lines"], for_oracle["anchors"], for_oracle["refs"], 0, 66, 69, 8)
+            assert st & O.ST_BAD_REF
+            assert sp[0].cpu().numpy().tolist() == ref.tolist()
+            assert status == ssa.DEV_BAD_REF
+            index, counts, status = run_refs_index(on_device, 96)
+            want = O.spans_to_index(ref, 69)
+            assert counts[0] == len(want) and index[0, :len(want)].tolist() == want.tolist()
+            assert status == ssa.DEV_BAD_REF
+
+
 @pytest.mark.parametrize("seed", range(5))
 def test_one_launch_fuzz(seed):
     reqs = fuzz_requests(seed + 100)
