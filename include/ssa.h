@@ -160,7 +160,9 @@ size_t ssa_decode_workspace_bytes(const ssa_attn_desc* desc, int32_t max_selecte
  *              also be page-locked host memory that the device addresses: a
  *              row then crosses the bus as soon as it is finished)
  *   workspace  dev, >= ssa_decode_workspace_bytes(desc, max_selected) bytes,
- *              16-byte aligned
+ *              16-byte aligned; always required (the size query never returns
+ *              0 for a valid descriptor, also when every request fits one
+ *              thread block and nothing is written to it)
  * Errors: SSA_ERR_NULL, SSA_ERR_SHAPE, SSA_ERR_DTYPE, SSA_ERR_ALIGN,
  * SSA_ERR_CAPACITY, SSA_ERR_WORKSPACE, SSA_ERR_UNSUPPORTED, SSA_ERR_CUDA.
  */
@@ -188,7 +190,8 @@ int32_t ssa_decode_attn_sparse(const ssa_attn_desc* desc, const void* q,
  *   max_spans     >= the number of spans of any request (a caller knows it: it
  *                 built the lists).  A request with more keeps its first
  *                 max_spans spans (SSA_DEV_TOO_MANY_SPANS).  Up to 128 spans
- *                 per request are merged on chip; with a larger bound (up to
+ *                 per request are merged on chip (up to 32 by every warp for
+ *                 itself, without a block barrier); with a larger bound (up to
  *                 SSA_MAX_SPANS_PER_SEQ, beyond which it is treated as that)
  *                 the call expands the lists with the kernel of
  *                 ssa_spans_to_index first and attends through them - two
@@ -201,7 +204,12 @@ int32_t ssa_decode_attn_sparse(const ssa_attn_desc* desc, const void* q,
  *   index_out   dev int32 [B * index_stride] or NULL; index_stride >=
  *               max_selected when given; entries past the count untouched
  *   counts_out  dev int32 [B] or NULL
- *   span_offsets, spans, ctx_lens  dev, as in ssa_spans_to_index
+ *   span_offsets, spans, ctx_lens  dev, as in ssa_spans_to_index.  span_offsets
+ *               may be NULL when max_spans <= 128: the lists are then a table
+ *               of exactly max_spans pairs per request (request b owns pairs
+ *               b*max_spans .. (b+1)*max_spans - 1, unused ones empty, e.g.
+ *               (0, 0) - the layout ssa_refs_to_spans writes), which saves the
+ *               blocks one dependent read (SSA_ERR_UNSUPPORTED above 128)
  *   workspace   dev, >= ssa_decode_spans_workspace_bytes(desc, max_selected,
  *               max_spans) bytes, 16-byte aligned, no initialisation needed
  * A paged cache is not supported by this call.
@@ -409,11 +417,30 @@ int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, cons
  * the attention kernels then store each finished row straight across the bus
  * while the rest of the batch is still being read, and the copy out only has
  * to carry what kernels also read back (counts, the status word).
+ *
+ * Which kernels run.  The lists index / counts are always written and the
+ * results are always those of the two calls, bit for bit.  When the caller
+ * states a bound on the spans per request (max_spans > 0) the step may run as
+ * ONE kernel instead - ssa_decode_attn_spans with index / counts as its
+ * optional outputs - which removes the index launch from short steps:
+ *   SSA_STEP_ONE_KERNEL   always (needs 0 < max_spans <= 128 and a workspace
+ *                         of ssa_decode_spans_workspace_bytes(desc,
+ *                         max_selected, max_spans) bytes, else
+ *                         SSA_ERR_CAPACITY / SSA_ERR_WORKSPACE)
+ *   SSA_STEP_TWO_KERNELS  never
+ *   neither               the library decides: one kernel when max_spans <= 32,
+ *                         the workspace suffices, the inputs are not fetched by
+ *                         kernel (that fetch is fused with the index launch)
+ *                         and the attention grid is at most four waves of
+ *                         thread blocks - where every block repeating the merge
+ *                         of its request's spans costs less than a launch.
  * Errors: SSA_ERR_NULL for a NULL desc/step or an inconsistent copy request,
- * SSA_ERR_UNSUPPORTED for unknown flag bits, otherwise those of the two calls;
- * nothing after a failing stage is enqueued.
+ * SSA_ERR_UNSUPPORTED for unknown or contradictory flag bits, otherwise those
+ * of the calls made; nothing after a failing stage is enqueued.
  */
 #define SSA_STEP_COPY_BY_KERNEL 1u
+#define SSA_STEP_ONE_KERNEL 2u
+#define SSA_STEP_TWO_KERNELS 4u
 typedef struct {
   const int32_t* span_offsets;  /* dev [B+1]                                   */
   const int32_t* spans;         /* dev (start, end) pairs                      */
@@ -436,7 +463,8 @@ typedef struct {
   void* host_out;               /* host (pinned) or NULL                       */
   const void* dev_out;          /* dev                                         */
   size_t out_bytes;
-  uint32_t flags;               /* 0 or SSA_STEP_COPY_BY_KERNEL                */
+  uint32_t flags;               /* OR of SSA_STEP_* bits                       */
+  int32_t max_spans;            /* host bound on spans per request; 0: unknown */
 } ssa_step;
 
 int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* step, void* stream);
@@ -462,7 +490,9 @@ int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* step, void* s
  *    with SSA_ERR_WORKSPACE and nothing is launched;
  *  - the first call on each device looks up the array's device address (the
  *    device must be current); make that first call outside any stream
- *    capture.  No call allocates or frees memory;
+ *    capture.  The address is kept per device ordinal for the device's
+ *    primary context (the one the runtime API uses) and is stale after
+ *    cudaDeviceReset.  No call allocates or frees memory;
  *  - all calls share the one array, and it keeps whatever the previous call
  *    left in it.  Nothing in it needs to start at zero (every slot is written
  *    before it is read within a call), but two calls whose kernels overlap on

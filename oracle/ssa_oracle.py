@@ -215,31 +215,33 @@ def encode_blocked(idx, bs: int):
 
 
 def attn_alg1_blocked(q, K, V, n: int, metadata, bs: int, scale: float):
-    """Algorithm 1 with the readings stated in the module header."""
-    D = V.shape[-1]
-    nb = (max(n, 0) + bs - 1) // bs
-    qK = np.full(nb * bs, -np.inf)            # unlisted blocks: excluded
-    for blk, bm in metadata:
-        soft = np.where(bm, 0.0, -np.inf)     # bit 1 -> +0, bit 0 -> -inf
-        delta = blk * bs
-        bqK = np.zeros(bs)
-        for i in range(bs):
-            if delta + i < n:
-                bqK[i] = float(np.dot(q, K[delta + i]))
-        qK[delta:delta + bs] = bqK + soft
-    Z = qK * scale
-    zmax = np.max(Z) if Z.size else -np.inf
-    if not np.isfinite(zmax):
-        return np.zeros(D), -np.inf
-    E = np.exp(Z - zmax)
-    A = E / np.sum(E)
-    o = np.zeros(D)
-    for blk, bm in metadata:
-        delta = blk * bs
-        for i in range(bs):
-            if delta + i < n and A[delta + i] != 0.0:
-                o += A[delta + i] * V[delta + i]
-    return o, float(zmax + np.log(np.sum(E)))
+    """Attention from the blocked span encoding, in the two phases of
+    Algorithm 1 (scores of the listed blocks, one softmax over the context,
+    weighted sum of the listed blocks' value rows), with the readings stated
+    in the module header.  ``metadata``: (block index, boolean mask of ``bs``
+    positions) pairs as ``encode_blocked`` returns them."""
+    n = max(int(n), 0)
+    scores = np.full(n, -np.inf)              # a position of no listed block stays excluded
+    listed = []
+    for block, mask in metadata:
+        first = int(block) * bs
+        inside = np.arange(first, min(first + bs, n))
+        listed.append(inside)
+        # every position of a listed block gets its score; the block's mask then
+        # leaves selected positions as they are and sends the others to -inf
+        penalty = np.where(np.asarray(mask, dtype=bool)[: len(inside)], 0.0, -np.inf)
+        scores[inside] = scale * (K[inside] @ q) + penalty
+    top = np.max(scores) if n else -np.inf
+    if not np.isfinite(top):
+        return np.zeros(V.shape[-1]), -np.inf
+    weights = np.exp(scores - top)
+    total = np.sum(weights)
+    weights = weights / total
+    out = np.zeros(V.shape[-1])
+    for inside in listed:                     # only listed blocks contribute value rows
+        live = inside[weights[inside] != 0.0]  # weight exactly zero: the row is not touched
+        out += weights[live] @ V[live]
+    return out, float(top + np.log(total))
 
 
 def resolve_references(lines, anchor_line, refs, prefix_len: int, line_start: int, ctx_len: int,

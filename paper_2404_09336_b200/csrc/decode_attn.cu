@@ -24,6 +24,7 @@
 // the request's span list itself, which the block sorts and merges in shared
 // memory and turns into positions by arithmetic (no index list anywhere).
 #include <algorithm>
+#include <atomic>
 #include <type_traits>
 
 #include "fetch_index.cuh"
@@ -151,6 +152,7 @@ decode_partial_kernel(const DecodeParams p) {
   __shared__ float s_m[kGroups], s_l[kGroups];
   __shared__ int s_wcount[kWarps];
   __shared__ typename std::conditional<kMode == kSpans, SpanRuns, int>::type s_runs;
+  __shared__ typename std::conditional<kMode == kSpans, WarpRuns, int>::type s_wruns[kMode == kSpans ? kWarps : 1];
 
   const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -187,17 +189,39 @@ decode_partial_kernel(const DecodeParams p) {
     qraw.w[4] = c4.x; qraw.w[5] = c4.y; qraw.w[6] = c4.z; qraw.w[7] = c4.w;
   }
 
+  // span lists: where the request's list is; with up to 32 spans every lane asks for "its" span right away (a
+  // fixed-stride table needs no offsets, so the spans then arrive together with the sizes and the query)
+  int span_first = 0, span_n = 0;
+  int2 my_span = make_int2(0, 0);
+  const bool warp_merge = kMode == kSpans && p.span_cap <= 32;
+  if constexpr (kMode == kSpans) {
+    if (p.span_offsets) {
+      span_first = __ldg(p.span_offsets + b);
+      span_n = __ldg(p.span_offsets + b + 1) - span_first;
+    } else {
+      span_first = b * p.span_cap;
+      span_n = p.span_cap;
+    }
+    if (warp_merge && lane < min(span_n, p.span_cap)) my_span = __ldg(p.spans + span_first + lane);
+  }
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
+  int warp_runs = 1;                                  // span_cap rounded up to a power of two
+  while (warp_merge && warp_runs < p.span_cap) warp_runs <<= 1;
   if constexpr (kMode == kSpans) {
     // the request's spans -> disjoint ascending runs in shared memory (every block of the request repeats this)
-    const int first = __ldg(p.span_offsets + b);
-    const int total = merge_spans_block<kThreads>(s_runs, p.spans + first, __ldg(p.span_offsets + b + 1) - first,
-                                                  p.span_cap, n);
+    int total;
+    if (warp_merge) {                                 // up to 32 spans: every warp merges them for itself, no barrier
+      int S = max(span_n, 0);
+      if (S > p.span_cap) { S = p.span_cap; flags |= SSA_DEV_TOO_MANY_SPANS; }
+      total = merge_spans_warp(s_wruns[warp], my_span, S, warp_runs, n, flags);
+    } else {
+      total = merge_spans_block<kThreads>(s_runs, p.spans + span_first, span_n, p.span_cap, n);
+      if (tid == 0) flags |= s_runs.flags;
+    }
     c = min(total, p.max_selected);
     if (total > p.max_selected) flags |= SSA_DEV_OVERFLOW;
-    if (tid == 0) flags |= s_runs.flags;
   }
   if (start >= c && chunk_id > 0) return;             // chunk 0 always reports
   int cnt = max(0, min(p.chunk, c - start));          // list entries of this block; rows, except for bitmasks
@@ -241,7 +265,7 @@ decode_partial_kernel(const DecodeParams p) {
     for (int j = 0; j < kIdxPerThread; ++j) {
       const int r = staged_row(lane + 32 * j);
       if (r < cnt) {
-        const int v = span_position(s_runs, start + r);
+        const int v = warp_merge ? span_position(s_wruns[warp], warp_runs, start + r) : span_position(s_runs, start + r);
         s_idx[r] = v;
         if (row) row[r] = v;
       }
@@ -441,15 +465,16 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   // The second pass costs about as much as two rounds of a block, so a request is split only when that buys
   // parallelism: one chunk whenever the list fits a block's staging area and either every SM gets a block or
   // the list is short anyway; otherwise 256-entry chunks, halved while the grid has under two blocks per SM.
-  const long long want = 148 * 2;
+  const long long sms = sm_count();
+  const long long want = sms * 2;
   int chunk = 256;
-  if (max_selected <= kMaxChunk && (units >= 148 || max_selected <= 256)) chunk = kMaxChunk;
+  if (max_selected <= kMaxChunk && (units >= sms || max_selected <= 256)) chunk = kMaxChunk;
   else while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
   if (shares_rows(d) && max_selected > kMaxChunk) {
     // The row-sharing kernel leaves G triples per chunk and its blocks are long: fewer, larger chunks
     // (its blocks walk a chunk in windows of the staging area).  About 2048 blocks for groups of up to 8
     // heads, one block per resident slot for larger groups (measured, B*H_kv = 64..256, context 8192).
-    const long long target = d->H / d->H_kv > 8 ? 148 * 2 : 2048;
+    const long long target = d->H / d->H_kv > 8 ? sms * 2 : 2048;
     long long n = target / units;                              // rounded down: never one block over a full wave
     n = std::max<long long>(1, std::min<long long>(n, (max_selected + 255) / 256));
     chunk = std::max(chunk, (int)(((max_selected + n - 1) / n + 63) / 64 * 64));
@@ -582,7 +607,7 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   }
   if (mode == kBlockMask && (!bl || !bl->block_idx || !bl->block_mask || !counts)) return SSA_ERR_NULL;
   if (mode == kSpans) {
-    if (!sl || !sl->span_offsets || !sl->spans) return SSA_ERR_NULL;
+    if (!sl || !sl->spans) return SSA_ERR_NULL;           // no offsets: a fixed-stride table
     if (pg) return SSA_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(sl->spans) % 8 != 0) return SSA_ERR_ALIGN;
   }
@@ -649,7 +674,7 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   // A grid of a few waves releases the next kernel at once (its blocks wait on
   // chip instead of being launched after the drain); a long grid does so only
   // as its blocks finish, so that waiting blocks do not crowd out its own.
-  p.early_release = (long long)d->B * d->H * pl.n_chunks <= 148ll * 4 * 6;
+  p.early_release = (long long)d->B * d->H * pl.n_chunks <= (long long)sm_count() * SSA_MIN_BLOCKS * 6;
   const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->D);
   p.scale_log2 = scale * kLog2e;
 
@@ -664,22 +689,38 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   return d->D == 128 ? launch<__half, 128>(p, d->B, mode, a32, st) : launch<__half, 64>(p, d->B, mode, a32, st);
 }
 
+int32_t one_kernel_span_limit() { return kDirectSpans; }
+
+// Every block of the span-list kernel repeats the merge of its request's spans (about a microsecond per wave
+// of blocks when a warp can do it alone), the index kernel does it once per request but costs a launch of its
+// own (3-4 us exposed).  Measured on the five workloads: one kernel wins or ties up to about four waves.
+bool one_kernel_step_pays(const ssa_attn_desc* d, int32_t max_selected, int32_t max_spans, size_t ws_bytes) {
+  Plan pl;
+  if (max_spans <= 0 || max_spans > 32 || !d || check_desc(d) != SSA_OK || !make_plan(d, max_selected, &pl))
+    return false;
+  if (ws_bytes < pl.total_bytes + counts_bytes(d)) return false;
+  const long long units = shares_rows(d) ? (long long)d->B * d->H_kv : (long long)d->B * d->H;
+  return units * pl.n_chunks <= 4ll * SSA_MIN_BLOCKS * sm_count();
+}
+
 // Scratch of ssa_decode_attn_sparse_noalloc: part of the library's device image.
 // In host code the name `g_static_scratch` is only a handle for
 // cudaGetSymbolAddress, never a device address to pass to a kernel.
 static __device__ __align__(256) unsigned char g_static_scratch[SSA_STATIC_SCRATCH_BYTES];
 
-// Device address of the array on the current device, looked up once per device.
+// Device address of the array on the current device (its primary context), looked up once per device; threads
+// that race on the first call all store the same value.  The address does not survive cudaDeviceReset.
 static void* static_scratch_address() {
-  static void* address[64] = {};
+  constexpr int kMaxDevices = 64;
+  static std::atomic<void*> address[kMaxDevices];
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!address[dev]) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
-    address[dev] = ptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  void* ptr = address[dev].load(std::memory_order_acquire);
+  if (!ptr) {
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return nullptr;
+    address[dev].store(ptr, std::memory_order_release);
   }
-  return address[dev];
+  return ptr;
 }
 
 }  // namespace ssa
@@ -690,11 +731,15 @@ int32_t ssa_decode_attn_sparse_noalloc(const ssa_attn_desc* desc, const void* q,
                                        const void* v_cache, const int32_t* ctx_lens, const int32_t* index,
                                        int32_t index_stride, const int32_t* counts, int32_t max_selected,
                                        void* out, float* lse, uint32_t* dev_status, void* stream) {
-  if (!desc) return SSA_ERR_NULL;
+  // the checks of ssa_decode_attn_sparse in its order, so that a bad call gets the same status from both
+  if (!desc || !q || !k_cache || !v_cache || !ctx_lens || !out || !index || !counts) return SSA_ERR_NULL;
   const int32_t rc = ssa::check_desc(desc);
   if (rc != SSA_OK) return rc;
+  if (index_stride <= 0 || max_selected <= 0 || max_selected > index_stride) return SSA_ERR_CAPACITY;
+  if (!ssa::aligned16(q) || !ssa::aligned16(k_cache) || !ssa::aligned16(v_cache) || !ssa::aligned16(out))
+    return SSA_ERR_ALIGN;
   ssa::Plan pl;
-  if (max_selected <= 0 || !ssa::make_plan(desc, max_selected, &pl)) return SSA_ERR_CAPACITY;
+  if (!ssa::make_plan(desc, max_selected, &pl)) return SSA_ERR_SHAPE;
   if (pl.total_bytes > SSA_STATIC_SCRATCH_BYTES) return SSA_ERR_WORKSPACE;   // beyond the built-in scratch
   void* scratch = ssa::static_scratch_address();
   if (!scratch) return SSA_ERR_CUDA;
@@ -721,8 +766,9 @@ int32_t ssa_decode_attn_spans(const ssa_attn_desc* desc, const void* q, const vo
                               int32_t max_spans, int32_t max_selected, void* out, float* lse, int32_t* index_out,
                               int32_t index_stride, int32_t* counts_out, void* workspace, size_t workspace_bytes,
                               uint32_t* dev_status, void* stream) {
-  if (!desc || !span_offsets || !spans) return SSA_ERR_NULL;
+  if (!desc || !spans) return SSA_ERR_NULL;
   if (max_spans <= 0) return SSA_ERR_CAPACITY;
+  if (!span_offsets && max_spans > ssa::kDirectSpans) return SSA_ERR_UNSUPPORTED;
   if (max_spans <= ssa::kDirectSpans) {
     const ssa::SpanLists sl = {span_offsets, spans, max_spans, index_out, counts_out};
     return ssa::run(desc, q, k_cache, v_cache, ctx_lens, nullptr, index_stride, nullptr, max_selected, out, lse,

@@ -103,9 +103,9 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   request_sizes(p, b, n, c, flags);
   if constexpr (kMode == kSpans) {
     // the request's spans -> disjoint ascending runs in shared memory
-    const int first = __ldg(p.span_offsets + b);
-    const int total = merge_spans_block<kThreads>(s_runs, p.spans + first, __ldg(p.span_offsets + b + 1) - first,
-                                                  p.span_cap, n);
+    const int first = p.span_offsets ? __ldg(p.span_offsets + b) : b * p.span_cap;
+    const int S = p.span_offsets ? __ldg(p.span_offsets + b + 1) - first : p.span_cap;
+    const int total = merge_spans_block<kThreads>(s_runs, p.spans + first, S, p.span_cap, n);
     c = min(total, p.max_selected);
     if (total > p.max_selected) flags |= SSA_DEV_OVERFLOW;
     if (tid == 0) flags |= s_runs.flags;

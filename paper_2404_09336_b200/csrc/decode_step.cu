@@ -29,7 +29,7 @@ static bool device_addressable_host(const void* p) {
 
 static int32_t copy_by_kernel(void* dst, const void* src, size_t bytes, cudaStream_t st) {
   const size_t n16 = bytes / 16;
-  const unsigned blocks = (unsigned)std::min<size_t>((n16 + 255) / 256, 148 * 4);
+  const unsigned blocks = (unsigned)std::min<size_t>((n16 + 255) / 256, (size_t)sm_count() * 4);
   const cudaError_t err = launch_pdl(copy_words_kernel, dim3(blocks), dim3(256), st, reinterpret_cast<uint4*>(dst),
                                      reinterpret_cast<const uint4*>(src), n16);
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
@@ -47,7 +47,9 @@ extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s,
   if (!desc || !s) return SSA_ERR_NULL;
   if (s->host_in && (!s->dev_in || s->in_bytes == 0)) return SSA_ERR_NULL;
   if (s->host_out && (!s->dev_out || s->out_bytes == 0)) return SSA_ERR_NULL;
-  if (s->flags & ~(uint32_t)SSA_STEP_COPY_BY_KERNEL) return SSA_ERR_UNSUPPORTED;
+  if (s->flags & ~(uint32_t)(SSA_STEP_COPY_BY_KERNEL | SSA_STEP_ONE_KERNEL | SSA_STEP_TWO_KERNELS))
+    return SSA_ERR_UNSUPPORTED;
+  if ((s->flags & SSA_STEP_ONE_KERNEL) && (s->flags & SSA_STEP_TWO_KERNELS)) return SSA_ERR_UNSUPPORTED;
   const bool by_kernel = (s->flags & SSA_STEP_COPY_BY_KERNEL) != 0;
   if (by_kernel) {                             // everything is checked before anything is enqueued
     if (s->host_in && !ssa::copy_aligned(s->host_in, s->dev_in, s->in_bytes)) return SSA_ERR_ALIGN;
@@ -67,7 +69,28 @@ extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s,
   const int32_t* h_off = by_kernel ? host_twin(s->span_offsets) : nullptr;
   const int32_t* h_spans = by_kernel ? host_twin(s->spans) : nullptr;
   const int32_t* h_ctx = by_kernel ? host_twin(s->ctx_lens) : nullptr;
-  if (h_off && h_spans && h_ctx && desc->B > 0 && desc->B < 60000) {
+  const bool fused_fetch = h_off && h_spans && h_ctx && desc->B > 0 && desc->B < 60000;
+  bool one_kernel = (s->flags & SSA_STEP_ONE_KERNEL) != 0;
+  if (one_kernel) {
+    if (s->max_spans <= 0 || s->max_spans > ssa::one_kernel_span_limit()) return SSA_ERR_CAPACITY;
+  } else if (!(s->flags & SSA_STEP_TWO_KERNELS) && !fused_fetch) {
+    one_kernel = ssa::one_kernel_step_pays(desc, s->max_selected, s->max_spans, s->workspace_bytes);
+  }
+  if (one_kernel) {
+    if (s->host_in) {
+      if (by_kernel) {
+        rc = ssa::copy_by_kernel(s->dev_in, s->host_in, s->in_bytes, st);
+        if (rc != SSA_OK) return rc;
+      } else if (cudaMemcpyAsync(s->dev_in, s->host_in, s->in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        return SSA_ERR_CUDA;
+      }
+    }
+    rc = ssa_decode_attn_spans(desc, s->q, s->k_cache, s->v_cache, s->ctx_lens, s->span_offsets, s->spans,
+                               s->max_spans, s->max_selected, s->out, s->lse, s->index, s->index_stride, s->counts,
+                               s->workspace, s->workspace_bytes, s->dev_status, stream);
+    if (rc != SSA_OK) return rc;
+  } else {
+  if (fused_fetch) {
     // the span lists are part of what is fetched: expand them straight from the host arena while the same
     // launch copies the arena in
     rc = ssa::fetch_and_index(h_off, h_spans, h_ctx, desc->B, s->index, s->index_stride, s->counts, s->dev_status,
@@ -90,6 +113,7 @@ extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s,
                               s->counts, s->max_selected, s->out, s->lse, s->workspace, s->workspace_bytes,
                               s->dev_status, stream);
   if (rc != SSA_OK) return rc;
+  }
   if (s->host_out) {
     if (by_kernel) {
       rc = ssa::copy_by_kernel(const_cast<void*>(s->host_out), s->dev_out, s->out_bytes, st);

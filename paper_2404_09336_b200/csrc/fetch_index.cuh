@@ -1,4 +1,4 @@
-// Internal entry points defined in spans_to_index.cu and used by decode_step.cu and decode_attn.cu.
+// Internal entry points shared between spans_to_index.cu, decode_attn.cu and decode_step.cu.
 #pragma once
 #include "ssa_common.cuh"
 
@@ -15,5 +15,10 @@ int32_t fetch_and_index(const int32_t* host_span_offsets, const int32_t* host_sp
 int32_t spans_to_index_capped(const int32_t* span_offsets, const int32_t* spans, const int32_t* ctx_lens, int32_t B,
                               int32_t* index, int32_t index_stride, int32_t capacity, int32_t span_cap,
                               int32_t* counts, uint32_t* dev_status, cudaStream_t stream);
+
+// Defined in decode_attn.cu, for ssa_decode_step: the most spans per request the span-list attention kernel
+// merges on chip, and whether a step is better served by that one kernel than by index + attention launches.
+int32_t one_kernel_span_limit();
+bool one_kernel_step_pays(const ssa_attn_desc* desc, int32_t max_selected, int32_t max_spans, size_t workspace_bytes);
 
 }  // namespace ssa

@@ -122,6 +122,69 @@ __device__ __forceinline__ int merge_spans_block(SpanRuns& r, const int2* __rest
   return r.offs[P];
 }
 
+// The same for up to 32 spans, done by ONE warp for itself: no block barrier and nothing shared with the other
+// warps of the block, so a warp can go on to its cache rows as soon as its own lanes are done.  Lane i ends up
+// owning run i of the sorted, trimmed list; the runs go to the warp's own `w`.
+struct WarpRuns {
+  int32_t start[32];                        // first position of run i that no earlier run covers
+  int32_t offs[33];                         // positions before run i; offs[32] = all positions
+};
+
+// Called by all 32 lanes.  Lane i < S holds span i of the request in `my_span`; S <= P, P a power of two <= 32 (the work grows with P, not with 32:
+// a request of the method names a handful of spans).  Returns the number of attended positions and ORs the
+// status bits of the list into `flags` (every lane gets the same bits).
+__device__ __forceinline__ int merge_spans_warp(WarpRuns& w, int2 my_span, int S, int P, int n, uint32_t& flags) {
+  const int lane = threadIdx.x & 31;
+  uint32_t f = 0;
+  int2 se = make_int2(kNoSpan, kNoSpan);
+  if (lane < S) se = clamp_span(my_span, n, f);
+  // rank of this lane's span among the starts (ties by lane), then hand every span to the lane of its rank
+  int rank = 0;
+  for (int j = 0; j < P; ++j) {
+    const int sj = __shfl_sync(0xffffffffu, se.x, j);
+    rank += (sj < se.x || (sj == se.x && j < lane)) ? 1 : 0;
+  }
+  if (lane < P) {
+    w.start[rank] = se.x;
+    w.offs[rank] = se.y;
+  }
+  __syncwarp();
+  const int s0 = lane < P ? w.start[lane] : kNoSpan;
+  const bool live = s0 != kNoSpan;
+  const int s = live ? s0 : 0, e = live ? w.offs[lane] : 0;
+  __syncwarp();
+  int mx = e;                               // running maximum of the ends up to and including this run
+  for (int d = 1; d < P; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, mx, d);
+    if (lane >= d) mx = max(mx, o);
+  }
+  const int prev = __shfl_up_sync(0xffffffffu, mx, 1);
+  const int ns = lane == 0 ? s : max(s, prev);
+  const int len = live ? max(e - ns, 0) : 0;
+  int sum = len;
+  for (int d = 1; d < P; d <<= 1) {
+    const int o = __shfl_up_sync(0xffffffffu, sum, d);
+    if (lane >= d) sum += o;
+  }
+  const int total = __shfl_sync(0xffffffffu, sum, P - 1);
+  if (lane < P) {
+    w.start[lane] = ns;
+    w.offs[lane] = sum - len;
+  }
+  if (lane == 0) w.offs[P] = total;
+  flags |= __reduce_or_sync(0xffffffffu, f);
+  __syncwarp();
+  return total;
+}
+
+// The k-th attended position (0 <= k < offs[P]) among P runs.
+__device__ __forceinline__ int span_position(const WarpRuns& w, int P, int k) {
+  int lo = 0;
+  for (int step = P >> 1; step > 0; step >>= 1)
+    if (w.offs[lo + step] <= k) lo += step;
+  return w.start[lo] + (k - w.offs[lo]);
+}
+
 // The k-th attended position (0 <= k < offs[P]): the last run i with offs[i] <= k holds it.
 __device__ __forceinline__ int span_position(const SpanRuns& r, int k) {
   int lo = 0, hi = r.P;

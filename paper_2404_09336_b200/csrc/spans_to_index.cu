@@ -227,7 +227,7 @@ int32_t fetch_and_index(const int32_t* host_span_offsets, const int32_t* host_sp
   const int32_t slice = (index_stride + slices - 1) / slices;
   const size_t n16 = bytes / 16;
   const size_t per_row = (size_t)slices * kIdxThreads * 2;            // two words per thread
-  const int copy_rows = (int)std::min<size_t>((n16 + per_row - 1) / per_row, 148 * 8);
+  const int copy_rows = (int)std::min<size_t>((n16 + per_row - 1) / per_row, (size_t)sm_count() * 8);
   if (B + copy_rows > 65535) return SSA_ERR_SHAPE;
   SpanSource s = {};
   s.span_offsets = host_span_offsets; s.spans = host_spans; s.ctx_lens = host_ctx_lens;

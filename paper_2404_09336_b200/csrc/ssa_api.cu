@@ -1,8 +1,30 @@
 // Library-wide entry points of libssa: status strings, version, the timing
 // hook and the launch counter.
+#include <atomic>
+
 #include "ssa_common.cuh"
 
 namespace ssa {
+
+// Multiprocessors of the current device, asked once per device.  Without a usable device (size queries on a
+// machine that has none) the count of a full B200 stands in.
+int sm_count() {
+  constexpr int kDefault = 148, kMaxDevices = 64;
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return kDefault;
+  }
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return kDefault;
+  }
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
 
 static thread_local uint64_t t_launches = 0;
 static thread_local cudaEvent_t t_ev_begin = nullptr;

@@ -16,6 +16,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 // Per-thread bookkeeping shared by the entry points (defined in ssa_api.cu).
 void note_launches(int n);
 void take_kernel_events(cudaEvent_t* begin, cudaEvent_t* end);
+int sm_count();   // multiprocessors of the current device (cached; no synchronisation)
 
 // Programmatic dependent launch.  Every kernel of the library is launched
 // with the programmatic-serialization attribute: its blocks may become

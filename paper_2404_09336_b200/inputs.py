@@ -230,6 +230,22 @@ def make_config(cfg: int, density: float | None = None, B: int | None = None, H:
     return _finish(name, seed, B, H, D, T, dtype, ctx, per_seq, first_id)
 
 
+def make_mixed(every: int, B: int | None = None, H: int | None = None, first_id: int = 0) -> Workload:
+    """Workload 2 with every ``every``-th request at a "determine span" step of
+    the method (Sec. "Self-selected attention span", Inference: such a step
+    attends to the whole preceding context): its list is the single span
+    [0, ctx_len); the other requests keep their selected spans."""
+    base = make_config(2, B=B, H=H, first_id=first_id)
+    per_seq = []
+    for i in range(base.B):
+        if i % every == 0:
+            per_seq.append([(0, int(base.ctx_lens[i]))])
+        else:
+            per_seq.append([tuple(int(x) for x in p) for p in base.spans_of(i)])
+    return _finish(f"mixed_every_{every}", base.seed, base.B, base.H, base.D, base.max_ctx, base.dtype,
+                   base.ctx_lens, per_seq, first_id)
+
+
 def make_microbench(ctx: int, sparsity_block: int, B: int = 64, H: int = 32, max_ctx: int | None = None,
                     first_id: int = 0) -> Workload:
     """The paper's kernel micro-benchmark (Sec. "Custom CUDA kernel

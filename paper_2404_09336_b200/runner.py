@@ -1,5 +1,5 @@
 """Device-side plumbing around the C-ABI calls: buffers for one workload and
-the two-call decode step (span list -> index list -> attention).
+the decode step (span lists -> index lists -> attention).
 
 Only allocation, host<->device copies and calls of ``ssa.*`` happen here.
 """
@@ -119,6 +119,7 @@ class DecodeStep:
         if need == 0:
             raise RuntimeError("ssa_decode_workspace_bytes rejected the descriptor")
         self.workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+        self._steps = {}
 
     def select_copy(self, c: int):
         ks, vs = self.k_store[c % len(self.k_store)], self.v_store[c % len(self.v_store)]
@@ -159,6 +160,7 @@ class DecodeStep:
         need = ssa.decode_blockmask_workspace_bytes(self.desc, block_size, self.block_stride)
         if need > self.workspace.numel():
             self.workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+            self._steps = {}
 
     def _bound_blocks(self):
         """Host-side bound on the listed blocks of any request: no more than its context spans."""
@@ -178,10 +180,23 @@ class DecodeStep:
         self.build_blockmask(stream)
         self.attend_blockmask(stream)
 
-    def step(self, stream=None):
-        """One decode step of the method: span lists -> index lists -> attention."""
+    def step_two_calls(self, stream=None):
+        """One decode step as two calls: span lists -> index lists -> attention."""
         self.build_index(stream)
         self.attend_sparse(stream)
+
+    def step(self, stream=None, kernels="auto"):
+        """One decode step of the method through ssa_decode_step with everything resident on the
+        device: index lists, counts and the attention output are written.  kernels: "auto" (the
+        library picks one kernel or index + attention launches), "one" or "two"."""
+        key = ("resident", self.k.data_ptr(), self.max_selected, self.max_spans, kernels)
+        st = self._steps.get(key)
+        if st is None:
+            st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q, self.k,
+                               self.v, self.max_selected, self.out, self.lse, self.workspace, self.status,
+                               max_spans=self.max_spans, kernels=kernels)
+            self._steps[key] = st
+        return ssa.decode_step(self.desc, st, stream)
 
     # ---- host-buffer form (end-to-end timing) -----------------------------------------
     def make_host_buffers(self):
@@ -189,7 +204,6 @@ class DecodeStep:
         context lengths, span lists) and a pinned landing buffer for what the
         caller reads back (output rows, lse, counts, status word).
         Returns (host-to-device bytes, device-to-host bytes) per step."""
-        self._host_steps = {}
         self.h_in = self.in_arena.cpu().pin_memory()
         self.h_out = torch.empty(self.out_arena.shape, dtype=torch.uint8).pin_memory()
         self.h_out_rows, self.h_lse, self.h_counts, self.h_status = _views(self.h_out, self._out_specs)
@@ -207,20 +221,22 @@ class DecodeStep:
         (SSA_STEP_COPY_BY_KERNEL).  Same bytes, same result, less latency."""
         if not hasattr(self, "h_in"):
             raise RuntimeError("call make_host_buffers() before step_from_host()")
-        key = (self.k.data_ptr(), self.max_selected, bool(direct))
-        st = self._host_steps.get(key)
+        key = ("host", self.k.data_ptr(), self.max_selected, self.max_spans, bool(direct))
+        st = self._steps.get(key)
         if st is None:
             if direct:
                 tail = self.counts.data_ptr() - self.out_arena.data_ptr()   # counts + status: kernels read them too
                 st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q,
                                    self.k, self.v, self.max_selected, self.h_out_rows, self.h_lse, self.workspace,
                                    self.status, host_in=self.h_in, dev_in=self.in_arena,
-                                   host_out=self.h_out[tail:], dev_out=self.out_arena[tail:], copy_by_kernel=True)
+                                   host_out=self.h_out[tail:], dev_out=self.out_arena[tail:], copy_by_kernel=True,
+                                   max_spans=self.max_spans)
             else:
                 st = ssa.make_step(self.span_offsets, self.spans, self.ctx_lens, self.index, self.counts, self.q,
                                    self.k, self.v, self.max_selected, self.out, self.lse, self.workspace, self.status,
-                                   host_in=self.h_in, dev_in=self.in_arena, host_out=self.h_out, dev_out=self.out_arena)
-            self._host_steps[key] = st
+                                   host_in=self.h_in, dev_in=self.in_arena, host_out=self.h_out, dev_out=self.out_arena,
+                                   max_spans=self.max_spans)
+            self._steps[key] = st
         return ssa.decode_step(self.desc, st, stream)
 
     def set_spans(self, wl: Workload):

@@ -45,7 +45,7 @@ class Step(C.Structure):
         ("dev_status", C.c_void_p), ("index_stride", C.c_int32), ("max_selected", C.c_int32),
         ("host_in", C.c_void_p), ("dev_in", C.c_void_p), ("in_bytes", C.c_size_t),
         ("host_out", C.c_void_p), ("dev_out", C.c_void_p), ("out_bytes", C.c_size_t),
-        ("flags", C.c_uint32),
+        ("flags", C.c_uint32), ("max_spans", C.c_int32),
     ]
 
 
@@ -326,12 +326,12 @@ def refs_to_spans(line_offsets, lines, anchor_offsets, anchor_line, ref_offsets,
     return _check("ssa_refs_to_spans", rc, check)
 
 
-STEP_COPY_BY_KERNEL = 1
+STEP_COPY_BY_KERNEL, STEP_ONE_KERNEL, STEP_TWO_KERNELS = 1, 2, 4
 
 
 def make_step(span_offsets, spans, ctx_lens, index, counts, q, k_cache, v_cache, max_selected, out, lse=None,
               workspace=None, dev_status=None, host_in=None, dev_in=None, host_out=None, dev_out=None,
-              copy_by_kernel=False) -> Step:
+              copy_by_kernel=False, max_spans=0, kernels="auto") -> Step:
     """Fill an ssa_step from tensors (addresses only; keep the tensors alive)."""
     addr = lambda t: None if t is None else t.data_ptr()
     nbytes = lambda t: 0 if t is None else t.numel() * t.element_size()
@@ -343,12 +343,14 @@ def make_step(span_offsets, spans, ctx_lens, index, counts, q, k_cache, v_cache,
     s.dev_status, s.index_stride, s.max_selected = addr(dev_status), _row_stride(index), int(max_selected)
     s.host_in, s.dev_in, s.in_bytes = addr(host_in), addr(dev_in), nbytes(host_in)
     s.host_out, s.dev_out, s.out_bytes = addr(host_out), addr(dev_out), nbytes(host_out)
-    s.flags = STEP_COPY_BY_KERNEL if copy_by_kernel else 0
+    s.flags = (STEP_COPY_BY_KERNEL if copy_by_kernel else 0) | {"auto": 0, "one": STEP_ONE_KERNEL,
+                                                                 "two": STEP_TWO_KERNELS}[kernels]
+    s.max_spans = int(max_spans)
     return s
 
 
 def decode_step(desc: AttnDesc, step: Step, stream=None, check=True):
-    """ssa_decode_step: [copy in] -> spans_to_index -> decode_attn_sparse -> [copy out], one call."""
+    """ssa_decode_step: [copy in] -> span lists to index lists and attention (one kernel or two) -> [copy out]."""
     return _check("ssa_decode_step", lib.ssa_decode_step(C.byref(desc), C.byref(step), _stream(stream)), check)
 
 

@@ -121,8 +121,10 @@ def test_step_rejects_bad_copy_requests_before_enqueuing_anything():
     st.host_in, st.dev_in, st.in_bytes = 0x1000, None, 256
     assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_NULL         # a copy without a destination
     st.dev_in = 0x2000
-    st.flags = 2
+    st.flags = 8
     assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_UNSUPPORTED  # unknown flag bit
+    st.flags = ssa.STEP_ONE_KERNEL | ssa.STEP_TWO_KERNELS
+    assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_UNSUPPORTED  # contradictory
     st.flags = ssa.STEP_COPY_BY_KERNEL
     st.host_in = 0x1008
     assert ssa.decode_step(d, st, stream=0, check=False) == ssa.ERR_ALIGN

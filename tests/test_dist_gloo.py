@@ -2,6 +2,7 @@
 request with no exchange on the data path, every rank's shard reproduces its
 part of the unsharded result, and the benchmark's reductions (time = max over
 ranks, bytes = sum over ranks) behave."""
+import json
 import os
 import socket
 import subprocess
@@ -76,3 +77,33 @@ def test_two_ranks_shard_the_batch(tmp_path):
         outs.append(o)
     assert all(p.returncode == 0 for p in procs), "\n".join(outs)
     assert "GLOO_OK" in outs[0]
+
+
+def test_bench_starts_its_own_ranks_when_run_as_a_plain_script():
+    """`python bench.py --gpus 2` without torchrun: the script re-launches itself as two ranks.  With
+    SSA_BENCH_DRY_RUN=1 the ranks use gloo and a stand-in measurement (rank r: 10 + r ms for
+    1000 * (r + 1) bytes per step), so the reductions can be checked: time = max, bytes = sum."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    env.update(SSA_BENCH_DRY_RUN="1", OMP_NUM_THREADS="1")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "20", "--warmup", "3"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stdout + res.stderr
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout                         # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["steps"] == 20 and line["dry_run"] is True
+    assert line["ms_per_step"] == 11.0 / 20                    # the slower rank's time
+    assert abs(line["value"] - 3000.0 * 20 / 11e-3 / 1e9) < 1e-12   # both ranks' bytes
+
+
+def test_clock_samples_between_the_first_and_last_region_count_as_under_load():
+    """Timed regions are far shorter than nvidia-smi's sampling period; the record must not come out empty."""
+    import bench
+    assert bench.host_cores() >= 1
+    rows = [(100.0 + 0.05 * i, "3996, 1965, 1965, 400.0, 0x0, Not Active, Not Active, Not Active, Active")
+            for i in range(40)]
+    # regions far shorter than the sampling period: every sample between the first and the last region counts
+    windows = [(100.5 + 0.001 * i, 100.5005 + 0.001 * i) for i in range(500)]
+    c = bench.summarize_clock_rows(rows, windows)
+    assert c["samples"] == 40 and c["samples_under_load"] >= 10
+    assert c["sm_mhz"] == 1965 and c["sm_max_mhz"] == 1965 and c["reasons"] == ["sw_power_cap"]

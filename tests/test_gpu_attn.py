@@ -477,7 +477,7 @@ def test_decode_step_in_one_call_with_host_copies():
     # ssa_decode_step: copy in, index, attention, copy out - against the two separate calls
     wl = inputs.make_config(2, B=5, H=4)
     ds = DecodeStep(wl, out_dtype=torch.float32)
-    ds.step()
+    ds.step_two_calls()
     torch.cuda.synchronize()
     want_out, want_lse = ds.out.clone(), ds.lse.clone()
     want_counts = ds.counts.clone()
@@ -489,7 +489,7 @@ def test_decode_step_in_one_call_with_host_copies():
     before = ssa.launch_count()
     ds.step_from_host()
     torch.cuda.synchronize()
-    assert ssa.launch_count() - before >= 2
+    assert ssa.launch_count() - before >= 1
     assert torch.equal(ds.out, want_out) and torch.equal(ds.lse, want_lse) and torch.equal(ds.counts, want_counts)
     host = ds.h_out.clone()
     assert torch.equal(host, ds.out_arena.cpu())               # results landed in the pinned arena
@@ -541,9 +541,49 @@ def test_decode_step_with_copies_done_by_kernels_and_rows_stored_into_host_memor
     st = mk(host_in=ds.h_in[8:264], dev_in=ds.in_arena, copy_by_kernel=True)
     assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_ALIGN
     st = mk(host_in=ds.h_in, dev_in=ds.in_arena)
-    st.flags = 6
+    st.flags = 8
     assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_UNSUPPORTED      # unknown flag bits
+    st.flags = ssa.STEP_ONE_KERNEL | ssa.STEP_TWO_KERNELS
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_UNSUPPORTED      # contradictory
     assert ssa.launch_count() == before
+
+
+@pytest.mark.parametrize("cfg,kw", [(2, dict(B=5, H=4)), (3, dict(B=2, H=3)), (5, dict(density=0.25, B=2, H=2))])
+def test_decode_step_runs_as_one_kernel_or_two_with_the_same_bits(cfg, kw):
+    """ssa_decode_step: forced to one kernel, forced to index + attention launches, and left to decide;
+    index lists, counts, output and lse agree bit for bit, and with the oracle."""
+    wl = inputs.make_config(cfg, **kw)
+    ds = DecodeStep(wl, out_dtype=torch.float32)
+    got = {}
+    for kernels in ("two", "one", "auto"):
+        ds.out.fill_(5.0)
+        ds.lse.fill_(5.0)
+        ds.index.fill_(-7)
+        ds.counts.fill_(-7)
+        before = ssa.launch_count()
+        ds.step(kernels=kernels)
+        torch.cuda.synchronize()
+        got[kernels] = (ds.out.clone(), ds.lse.clone(), ds.index.clone(), ds.counts.clone(),
+                        ssa.launch_count() - before)
+        assert int(ds.status.item()) == 0
+    chunks = got["two"][4] - 1                                  # attention launches of the two-kernel form
+    assert got["one"][4] == chunks                              # the same without the index launch
+    assert got["auto"][4] in (chunks, chunks + 1)
+    for kernels in ("one", "auto"):
+        for a, b in zip(got[kernels][:4], got["two"][:4]):
+            assert torch.equal(a, b)
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, ds.index_stride)
+    assert got["one"][3].cpu().numpy().tolist() == counts.tolist()
+    for b in range(wl.B):
+        assert np.array_equal(got["one"][2][b, :counts[b]].cpu().numpy(), index[b, :counts[b]])
+    ref, _ = O.decode_attn_sparse(wl.q_bits(), *wl.kv_bits(), wl.ctx_lens, index, counts, scale_of(wl.D), wl.dtype)
+    assert_parity(got["one"][0].double().cpu().numpy(), ref, False, "one-kernel step")
+    # forcing one kernel without a usable span bound is refused
+    st = ssa.make_step(ds.span_offsets, ds.spans, ds.ctx_lens, ds.index, ds.counts, ds.q, ds.k, ds.v,
+                       ds.max_selected, ds.out, ds.lse, ds.workspace, ds.status, kernels="one", max_spans=0)
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_CAPACITY
+    st.max_spans = 129
+    assert ssa.decode_step(ds.desc, st, check=False) == ssa.ERR_CAPACITY
 
 
 def test_side_stream_graph_replay_and_determinism():

@@ -155,6 +155,51 @@ def test_empty_one_token_overlapping_unsorted_clipped(dtype, D):
     assert check_spans(p, lists[3:4] * 8, [64] * 8, 32, want_lists=False) == 1
 
 
+@pytest.mark.parametrize("stride", [1, 7, 32, 33, 128])
+def test_fixed_stride_table_without_offsets(stride):
+    """span_offsets = NULL: request b owns `stride` pairs of the table, unused ones empty."""
+    B, H, T, D = 5, 3, 900, 128
+    p = Problem(B, H, T, D, "bf16", seed=30 + stride)
+    rng = np.random.default_rng(stride)
+    ctx = [900, 17, 500, 900, 64]
+    table = np.zeros((B, stride, 2), np.int32)
+    lists = []
+    for b in range(B):
+        k = int(rng.integers(0, stride + 1)) if b else stride          # request 0 uses every slot
+        sp = [(int(a), int(a + rng.integers(0, 40))) for a in rng.integers(-3, ctx[b], size=k)]
+        slots = rng.permutation(stride)[:k]                              # padding anywhere in the row
+        for slot, pair in zip(slots, sp):
+            table[b, slot] = pair
+        lists.append([tuple(int(x) for x in row) for row in table[b]])
+    max_selected = 900
+    d_tab = torch.from_numpy(table).to(DEV)
+    d_ctx = torch.tensor(ctx, dtype=torch.int32, device=DEV)
+    index = torch.full((B, 928), -7, dtype=torch.int32, device=DEV)
+    counts = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+    out = torch.full((B, H, D), 777.0, dtype=torch.float32, device=DEV)
+    lse = torch.full((B, H), 777.0, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    desc = ssa.make_desc(p.q, p.k, p.v, out)
+    ws = torch.empty(ssa.decode_spans_workspace_bytes(desc, max_selected, stride), dtype=torch.uint8, device=DEV)
+    ssa.decode_attn_spans(desc, p.q, p.k, p.v, d_ctx, None, d_tab, stride, max_selected, out, lse, index, counts, ws,
+                          status)
+    torch.cuda.synchronize()
+    want_status = 0
+    ref_index = np.full((B, max_selected), -1, np.int32)
+    ref_counts = np.zeros(B, np.int32)
+    for b in range(B):
+        want_status |= O.spans_status(lists[b], ctx[b], max_selected)
+        idx = O.spans_to_index(lists[b], ctx[b])
+        ref_index[b, :len(idx)], ref_counts[b] = idx, len(idx)
+        assert int(counts[b]) == len(idx) and index[b, :len(idx)].cpu().numpy().tolist() == idx.tolist()
+    assert int(status.item()) == sum(v for k, v in GPU_BITS.items() if want_status & k)
+    ref, ref_lse = O.decode_attn_sparse(p.q_bits, p.k_bits, p.v_bits, np.asarray(ctx), ref_index, ref_counts,
+                                        1.0 / np.sqrt(D), "bf16")
+    live = ref_counts > 0
+    assert_parity(out.double().cpu().numpy(), ref, False, "fixed-stride table")
+    np.testing.assert_allclose(lse.double().cpu().numpy()[live], ref_lse[live], rtol=1e-5, atol=1e-5)
+
+
 def test_more_than_32_and_more_than_128_spans():
     B, H, T, D = 3, 2, 3000, 128
     p = Problem(B, H, T, D, "bf16", seed=4)
@@ -272,11 +317,12 @@ def test_argument_checks_launch_nothing():
     ctx = torch.tensor([64], dtype=torch.int32, device=DEV)
     ws = torch.empty(ssa.decode_spans_workspace_bytes(desc, 64, 1), dtype=torch.uint8, device=DEV)
     idx = torch.zeros((1, 32), dtype=torch.int32, device=DEV)
-    call = lambda **kw: ssa.decode_attn_spans(desc, p.q, p.k, p.v, ctx, kw.get("off", off), sp, kw.get("ms", 1),
+    call = lambda **kw: ssa.decode_attn_spans(desc, p.q, p.k, p.v, ctx, kw.get("off", off), kw.get("sp", sp), kw.get("ms", 1),
                                               kw.get("sel", 64), out, None, kw.get("idx"), None, kw.get("ws", ws),
                                               None, check=False)
     before = ssa.launch_count()
-    assert call(off=None) == ssa.ERR_NULL
+    assert call(sp=None) == ssa.ERR_NULL
+    assert call(off=None, ms=129) == ssa.ERR_UNSUPPORTED    # a fixed-stride table holds at most 128 pairs per request
     assert call(ms=0) == ssa.ERR_CAPACITY
     assert call(sel=0) == ssa.ERR_CAPACITY
     assert call(idx=idx) == ssa.ERR_CAPACITY            # list pitch 32 below max_selected 64
