@@ -37,6 +37,9 @@ What is stated here, and where the paper defines it:
                           attended, the line being generated attends to itself).
                           The paper gives no algorithm; the rules are stated in
                           the function.
+* ``decode_attn_sparse_multiq``  several query rows per head over one
+                          selected set (outside the paper, which decodes one
+                          token per step): the set form applied row by row.
 * ``merge_partials``      recombination of (max, sum, accumulator) partial
                           results of disjoint subsets; not in the paper (its
                           kernel runs one thread block per head and request),
@@ -386,6 +389,32 @@ def decode_attn_sparse(q, k_cache, v_cache, ctx_lens, index, counts, scale,
             o, e = attn_set_form(qv, Ks, Vs, np.arange(len(idx)), scale)
             out[b, h] = o
             lse[b, h] = e
+    return out, lse
+
+
+def decode_attn_sparse_multiq(q, k_cache, v_cache, ctx_lens, index, counts, scale, dtype: str = "bf16"):
+    """Several query tokens per request and head in one step, all attending
+    to the request's one selected set (the paper decodes one token per step,
+    "Token generation"; with several, every query row is its own instance of
+    the Background equations over the same mask row).
+
+    q[B, H, Tq, D]; cache, lists and conventions as ``decode_attn_sparse``;
+    query heads may outnumber cache heads (head h reads cache head
+    h // (H / H_kv)).  Returns out[B, H, Tq, D] and lse[B, H, Tq]."""
+    B, H, Tq, D = q.shape
+    group = H // np.asarray(k_cache).shape[1]
+    out = np.full((B, H, Tq, D), np.nan)
+    lse = np.full((B, H, Tq), np.nan)
+    for b in range(B):
+        n = int(ctx_lens[b])
+        idx = np.asarray(index[b][: int(counts[b])], dtype=np.int64)
+        idx = idx[(idx >= 0) & (idx < n)]
+        for h in range(H):
+            Ks = _as_f64(np.asarray(k_cache[b, h // group])[idx], dtype)
+            Vs = _as_f64(np.asarray(v_cache[b, h // group])[idx], dtype)
+            for t in range(Tq):
+                out[b, h, t], lse[b, h, t] = attn_set_form(_as_f64(q[b, h, t], dtype), Ks, Vs,
+                                                           np.arange(len(idx)), scale)
     return out, lse
 
 
