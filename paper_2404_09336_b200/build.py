@@ -14,6 +14,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libssa.so")
+PROBE_SRC = os.path.join(HERE, "probe", "gather_probe.cu")
+PROBE_LIB = os.path.join(HERE, "libssa_probe.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -50,7 +52,24 @@ def build_library(force: bool = False, defines=(), out: str = LIB, verbose: bool
     return out
 
 
+def build_probe(force: bool = False) -> str:
+    """The gather micro-benchmark (bench.py --probe gather): a library of its own, not part of libssa."""
+    if not force and not _stale(PROBE_LIB, [PROBE_SRC]):
+        return PROBE_LIB
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    if not os.path.exists(nvcc):
+        raise RuntimeError("nvcc not found: libssa_probe.so cannot be built")
+    tmp = PROBE_LIB + f".tmp{os.getpid()}"
+    res = subprocess.run([nvcc, *NVCC_FLAGS, "-o", tmp, PROBE_SRC], capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    os.replace(tmp, PROBE_LIB)
+    return PROBE_LIB
+
+
 if __name__ == "__main__":
     args = sys.argv[1:]
     out = args[args.index("-o") + 1] if "-o" in args else LIB
     build_library(force=True, defines=[a for a in args if a.startswith("-D")], out=out, verbose=True)
+    if "-o" not in args:
+        build_probe(force=True)
