@@ -283,6 +283,38 @@ int32_t ssa_decode_attn_dense_paged(const ssa_attn_desc* desc, const void* q, co
                                     size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /*
+ * Several query tokens per request in one step (the paper decodes one token
+ * per step, Sec. "Self-selected attention span", Token generation; this has
+ * no counterpart there - it is what speculative or multi-token decoding
+ * needs): n_q query rows per head, all attending to the request's ONE
+ * selected set, each row its own instance of the Background equations over
+ * the same mask row.  Row t of head h is at q + b*q_stride_b + h*q_stride_h +
+ * t*q_stride_t, its output at out + b*o_stride_b + h*o_stride_h +
+ * t*o_stride_t, its lse at lse[(b*H + h)*n_q + t].  The rows of one head
+ * must lie side by side: desc->q_stride_h == n_q*q_stride_t and
+ * desc->o_stride_h == n_q*o_stride_t (q and out laid out [B, H, n_q, D]),
+ * else SSA_ERR_UNSUPPORTED.  Everything else - desc, cache, lists, counts,
+ * status bits, errors - is as for ssa_decode_attn_sparse /
+ * ssa_decode_attn_dense.  The (head, token) pairs that share a K/V head are
+ * served like grouped query heads: while (H/H_kv)*n_q <= 16 and D = 128
+ * every selected row is read once for all of them.  H*n_q <= 65535.
+ * Workspace: ssa_decode_multiq_workspace_bytes(desc, n_q, max_selected)
+ * (max_selected = desc->max_ctx for the dense call).
+ */
+size_t ssa_decode_multiq_workspace_bytes(const ssa_attn_desc* desc, int32_t n_q, int32_t max_selected);
+int32_t ssa_decode_attn_sparse_multiq(const ssa_attn_desc* desc, int32_t n_q, int64_t q_stride_t,
+                                      int64_t o_stride_t, const void* q, const void* k_cache,
+                                      const void* v_cache, const int32_t* ctx_lens, const int32_t* index,
+                                      int32_t index_stride, const int32_t* counts, int32_t max_selected,
+                                      void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                      uint32_t* dev_status, void* stream);
+int32_t ssa_decode_attn_dense_multiq(const ssa_attn_desc* desc, int32_t n_q, int64_t q_stride_t,
+                                     int64_t o_stride_t, const void* q, const void* k_cache,
+                                     const void* v_cache, const int32_t* ctx_lens, void* out, float* lse,
+                                     void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                     void* stream);
+
+/*
  * Anchors and references -> span lists: the step before ssa_spans_to_index
  * (Sec. "Self-selected attention span": anchors identify groups of contiguous
  * tokens, the model names the anchors it needs, generation attends to the

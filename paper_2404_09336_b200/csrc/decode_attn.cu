@@ -797,6 +797,52 @@ int32_t ssa_decode_attn_spans(const ssa_attn_desc* desc, const void* q, const vo
                   pl.total_bytes, dev_status, stream, ssa::kIndex);
 }
 
+// Several query tokens per head: (head, token) pairs become the heads of a wider descriptor over the same cache
+// heads, so that the kernel for grouped query heads reads every selected row once for all of them.
+static int32_t widen_for_tokens(const ssa_attn_desc* desc, int32_t n_q, int64_t q_stride_t, int64_t o_stride_t,
+                                ssa_attn_desc* wide) {
+  if (!desc) return SSA_ERR_NULL;
+  if (n_q <= 0 || (long long)desc->H * n_q > 65535) return SSA_ERR_SHAPE;
+  if (desc->q_stride_h != (int64_t)n_q * q_stride_t || desc->o_stride_h != (int64_t)n_q * o_stride_t)
+    return SSA_ERR_UNSUPPORTED;                          // the rows of one head must lie side by side
+  *wide = *desc;
+  wide->H = desc->H * n_q;
+  wide->q_stride_h = q_stride_t;
+  wide->o_stride_h = o_stride_t;
+  return SSA_OK;
+}
+
+size_t ssa_decode_multiq_workspace_bytes(const ssa_attn_desc* desc, int32_t n_q, int32_t max_selected) {
+  ssa_attn_desc wide;
+  if (!desc || widen_for_tokens(desc, n_q, desc->q_stride_h / (n_q > 0 ? n_q : 1),
+                                desc->o_stride_h / (n_q > 0 ? n_q : 1), &wide) != SSA_OK)
+    return 0;
+  return ssa_decode_workspace_bytes(&wide, max_selected);
+}
+
+int32_t ssa_decode_attn_sparse_multiq(const ssa_attn_desc* desc, int32_t n_q, int64_t q_stride_t, int64_t o_stride_t,
+                                      const void* q, const void* k_cache, const void* v_cache,
+                                      const int32_t* ctx_lens, const int32_t* index, int32_t index_stride,
+                                      const int32_t* counts, int32_t max_selected, void* out, float* lse,
+                                      void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream) {
+  ssa_attn_desc wide;
+  const int32_t rc = widen_for_tokens(desc, n_q, q_stride_t, o_stride_t, &wide);
+  if (rc != SSA_OK) return rc;
+  return ssa::run(&wide, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out, lse,
+                  workspace, workspace_bytes, dev_status, stream, ssa::kIndex);
+}
+
+int32_t ssa_decode_attn_dense_multiq(const ssa_attn_desc* desc, int32_t n_q, int64_t q_stride_t, int64_t o_stride_t,
+                                     const void* q, const void* k_cache, const void* v_cache,
+                                     const int32_t* ctx_lens, void* out, float* lse, void* workspace,
+                                     size_t workspace_bytes, uint32_t* dev_status, void* stream) {
+  ssa_attn_desc wide;
+  const int32_t rc = widen_for_tokens(desc, n_q, q_stride_t, o_stride_t, &wide);
+  if (rc != SSA_OK) return rc;
+  return ssa::run(&wide, q, k_cache, v_cache, ctx_lens, nullptr, 0, nullptr, 0, out, lse, workspace,
+                  workspace_bytes, dev_status, stream, ssa::kDense);
+}
+
 size_t ssa_decode_blockmask_workspace_bytes(const ssa_attn_desc* desc, int32_t block_size, int32_t max_blocks) {
   ssa::Plan pl;
   if (!desc || ssa::check_desc(desc) != SSA_OK || !ssa::make_plan_blockmask(desc, block_size, max_blocks, &pl))

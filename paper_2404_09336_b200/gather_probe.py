@@ -91,7 +91,7 @@ def main():
                             "in_flight_per_sm_kb": blocks_per_sm * 4 * 8, "us": round(us, 1),
                             "gbs": round(nbytes / us / 1e3)})
         for copy_rows in sorted({1, run_rows}):
-            for blocks_per_sm, stages in ((1, 27), (2, 13), (4, 6), (8, 2)):
+            for blocks_per_sm, stages in ((1, 27), (2, 13), (4, 6), (8, 2), (8, 3), (16, 1)):
                 got = checksum_of(1, lists[0], sms * blocks_per_sm, stages, copy_rows)
                 if got != want or int(error.item()) != 0:
                     raise SystemExit(f"bulk-copy gather disagrees with the plain loads (run {run_rows}, copies of "

@@ -85,6 +85,14 @@ def _load():
     lib.ssa_decode_attn_spans.restype = C.c_int32
     lib.ssa_decode_attn_spans.argtypes = [C.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, C.c_int32, C.c_int32, vp, vp,
                                           vp, C.c_int32, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_multiq_workspace_bytes.restype = C.c_size_t
+    lib.ssa_decode_multiq_workspace_bytes.argtypes = [C.POINTER(AttnDesc), C.c_int32, C.c_int32]
+    lib.ssa_decode_attn_sparse_multiq.restype = C.c_int32
+    lib.ssa_decode_attn_sparse_multiq.argtypes = [C.POINTER(AttnDesc), C.c_int32, C.c_int64, C.c_int64, vp, vp, vp, vp,
+                                                  vp, C.c_int32, vp, C.c_int32, vp, vp, vp, C.c_size_t, vp, vp]
+    lib.ssa_decode_attn_dense_multiq.restype = C.c_int32
+    lib.ssa_decode_attn_dense_multiq.argtypes = [C.POINTER(AttnDesc), C.c_int32, C.c_int64, C.c_int64, vp, vp, vp, vp,
+                                                 vp, vp, vp, C.c_size_t, vp, vp]
     lib.ssa_spans_to_blockmask.restype = C.c_int32
     lib.ssa_spans_to_blockmask.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp, vp, C.c_int32, vp, vp, vp]
     lib.ssa_decode_blockmask_workspace_bytes.restype = C.c_size_t
@@ -217,6 +225,39 @@ def decode_attn_spans(desc, q, k_cache, v_cache, ctx_lens, span_offsets, spans, 
                                    _ptr(lse), _ptr(index_out), _row_stride(index_out) if index_out is not None else 0,
                                    _ptr(counts_out), _ptr(workspace), ws_bytes, _ptr(dev_status), _stream(stream))
     return _check("ssa_decode_attn_spans", rc, check)
+
+
+def make_desc_multiq(q, k_cache, v_cache, out, max_ctx=None, scale: float = 0.0):
+    """Descriptor for q[B,H,Tq,D], out[B,H,Tq,D] (several query tokens per head) over k_cache/v_cache[B,H_kv,T,D].
+    Returns (desc, n_q, q_stride_t, o_stride_t)."""
+    d = make_desc(q[:, :, 0], k_cache, v_cache, out[:, :, 0], max_ctx, scale)
+    return d, int(q.shape[2]), int(q.stride(2)), int(out.stride(2))
+
+
+def decode_multiq_workspace_bytes(desc: AttnDesc, n_q: int, max_selected: int) -> int:
+    return int(lib.ssa_decode_multiq_workspace_bytes(C.byref(desc), int(n_q), int(max_selected)))
+
+
+def decode_attn_sparse_multiq(desc, n_q, q_stride_t, o_stride_t, q, k_cache, v_cache, ctx_lens, index, counts,
+                              max_selected, out, lse=None, workspace=None, dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_sparse_multiq: n_q query rows per head over one selected set; out / lse are written."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_sparse_multiq(C.byref(desc), int(n_q), int(q_stride_t), int(o_stride_t), _ptr(q),
+                                           _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens), _ptr(index),
+                                           _row_stride(index) if index is not None else 0, _ptr(counts),
+                                           int(max_selected), _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes,
+                                           _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_sparse_multiq", rc, check)
+
+
+def decode_attn_dense_multiq(desc, n_q, q_stride_t, o_stride_t, q, k_cache, v_cache, ctx_lens, out, lse=None,
+                             workspace=None, dev_status=None, stream=None, check=True):
+    """ssa_decode_attn_dense_multiq: n_q query rows per head over the full context."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.ssa_decode_attn_dense_multiq(C.byref(desc), int(n_q), int(q_stride_t), int(o_stride_t), _ptr(q),
+                                          _ptr(k_cache), _ptr(v_cache), _ptr(ctx_lens), _ptr(out), _ptr(lse),
+                                          _ptr(workspace), ws_bytes, _ptr(dev_status), _stream(stream))
+    return _check("ssa_decode_attn_dense_multiq", rc, check)
 
 
 def spans_to_blockmask(span_offsets, spans, ctx_lens, block_size, block_idx, block_mask, block_counts,
