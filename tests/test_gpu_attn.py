@@ -91,7 +91,8 @@ def test_cfg5_reduced(f):
 
 
 # ---- full sizes, in the launch configuration the benchmark times; sampled outputs -----
-@pytest.mark.parametrize("cfg,density", [(2, None), (3, None), (4, None), (5, 0.05), (5, 0.50)])
+@pytest.mark.parametrize("cfg,density", [(2, None), (3, None), (4, None), (5, 0.01), (5, 0.05), (5, 0.10), (5, 0.25),
+                                         (5, 0.50), (5, 1.00)])
 def test_full_size_sampled(cfg, density):
     wl = inputs.make_config(cfg, density=density)
     rng = np.random.default_rng(cfg)
