@@ -471,10 +471,10 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   if (max_selected <= kMaxChunk && (units >= sms || max_selected <= 256)) chunk = kMaxChunk;
   else while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
   if (shares_rows(d) && max_selected > kMaxChunk) {
-    // The row-sharing kernel leaves G triples per chunk and its blocks are long: fewer, larger chunks
-    // (its blocks walk a chunk in windows of the staging area).  About 2048 blocks for groups of up to 8
-    // heads, one block per resident slot for larger groups (measured, B*H_kv = 64..256, context 8192).
-    const long long target = d->H / d->H_kv > 8 ? sms * 2 : 2048;
+    // The row-sharing kernel leaves G triples per chunk, its blocks stream (a ring of tiles per warp) and two of
+    // them fit an SM: about one block per resident slot, i.e. as few chunks as keep the SMs busy (measured,
+    // B*H_kv = 64..256, context 8192: within 3 % of the best split for groups of 4, 8 and 16 heads).
+    const long long target = sms * 2;
     long long n = target / units;                              // rounded down: never one block over a full wave
     n = std::max<long long>(1, std::min<long long>(n, (max_selected + 255) / 256));
     chunk = std::max(chunk, (int)(((max_selected + n - 1) / n + 63) / 64 * 64));
@@ -526,24 +526,19 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
   void (*kernel)(const DecodeParams);
   const bool share = D == 128 && p.kv_group >= 2 && p.kv_group <= kGqaHeads && mode != kBlockMask;
+  size_t dynamic_smem = 0;
   if (share) {
     grid.y = (unsigned)(p.H / p.kv_group);              // one block per K/V head
     const bool hi = p.kv_group > 8;
     if (mode == kIndex)
-      kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kIndex, true, true>
-                               : decode_partial_gqa_kernel<T, kIndex, true, false>)
-                  : (aligned32 ? decode_partial_gqa_kernel<T, kIndex, false, true>
-                               : decode_partial_gqa_kernel<T, kIndex, false, false>);
+      kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true> : decode_partial_gqa_kernel<T, kIndex, false>;
     else if (mode == kSpans)
-      kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kSpans, true, true>
-                               : decode_partial_gqa_kernel<T, kSpans, true, false>)
-                  : (aligned32 ? decode_partial_gqa_kernel<T, kSpans, false, true>
-                               : decode_partial_gqa_kernel<T, kSpans, false, false>);
+      kernel = hi ? decode_partial_gqa_kernel<T, kSpans, true> : decode_partial_gqa_kernel<T, kSpans, false>;
     else
-      kernel = hi ? (aligned32 ? decode_partial_gqa_kernel<T, kDense, true, true>
-                               : decode_partial_gqa_kernel<T, kDense, true, false>)
-                  : (aligned32 ? decode_partial_gqa_kernel<T, kDense, false, true>
-                               : decode_partial_gqa_kernel<T, kDense, false, false>);
+      kernel = hi ? decode_partial_gqa_kernel<T, kDense, true> : decode_partial_gqa_kernel<T, kDense, false>;
+    dynamic_smem = kStagedSmemBytes;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStagedSmemBytes) != cudaSuccess)
+      return SSA_ERR_CUDA;
   } else if (mode == kIndex && p.page_table)
     kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true, true>
                        : decode_partial_kernel<T, D, kIndex, false, true>;
@@ -556,7 +551,7 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   else
     kernel = aligned32 ? decode_partial_kernel<T, D, kDense, true> : decode_partial_kernel<T, D, kDense, false>;
   if (ev_b) cudaEventRecord(ev_b, st);
-  cudaError_t err = launch_pdl(kernel, grid, dim3(kThreads), st, p);
+  cudaError_t err = launch_pdl_smem(kernel, grid, dim3(kThreads), dynamic_smem, st, p);
   if (ev_e) cudaEventRecord(ev_e, st);
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   int launches = 1;

@@ -1,6 +1,7 @@
 // Pass 1 of the decode attention for grouped query heads (G = H / H_kv query
-// heads share one K/V head, 2 <= G <= 16, D = 128): one block per (chunk,
-// K/V head, request) reads every selected row ONCE and serves all G heads.
+// heads share one K/V head, 2 <= G <= 16, D = 128; also several query tokens
+// per head, which are served the same way): one block per (chunk, K/V head,
+// request) reads every selected row ONCE and serves all G heads.
 //
 // With G heads per row the work per byte is G times that of multi-head
 // attention and the packed-FMA path of decode_partial_kernel runs out of issue
@@ -8,18 +9,23 @@
 // to the tensor cores.  The shapes are far too small for tcgen05 tiles (G x 16
 // rows x 128), so they are warp-level mma.sync.m16n8k16 (16-bit inputs, fp32
 // accumulation) with the M dimension holding the query heads:
-//   S[16 heads, 16 rows]  = Q[16, 128] . K_tile^T          (2 x 8 mma)
-//   O[16 heads, 128 dims] += P[16, 16] . V_tile[16, 128]   (16 mma, twice)
-// Operands come straight from global memory into the fragment registers, no
-// shared-memory staging and no ldmatrix: a dot product does not care in which
-// order the dimensions are visited, so the k index of the mma is mapped to
-// the head dimension such that every lane needs CONTIGUOUS bytes of a row:
-//   Q/K:  lane (g = lane/4, j = lane%4) holds dims [32j, 32j+32) of head g
-//         (and g+8) / of row g of each 8-row half of the tile; k-step s uses
-//         its dims 32j+4s .. 32j+4s+3.
-//   V:    lane (g, j) holds dims [16g, 16g+16) of tile rows 2j, 2j+1, 2j+8,
-//         2j+9; n-tile u takes dim 16g+u, the two rows of a k pair are
-//         interleaved with one byte-permute each.
+//   S[16 heads, 16 rows]  = Q . K_tile^T : A = Q (registers, loaded once),
+//                           B = K tile via ldmatrix (rows are the n index);
+//   O[16 heads, 128 dims] += P . V_tile  : A = P from the accumulators of S,
+//                           B = V tile via ldmatrix.trans (rows are the k index).
+// The rows travel global -> shared memory by asynchronous 16-byte copies
+// (cp.async, evict-first in L2) into a ring of tiles that every warp keeps for
+// itself, and the fragments come out of that ring with ldmatrix.  The bytes in
+// flight are set by the ring (three tiles of 16 rows x (K + V) = 24 KB per
+// warp, 96 KB per block, two blocks per SM), not by fragment registers, and a
+// warp works on one tile while its next two are on their way; no block
+// barrier inside the tile loop.  (An earlier version loaded the fragments
+// straight from global memory into registers, one tile in flight per warp:
+// 5-15 % slower on long lists.)
+//
+// Shared-memory tiles are [16 rows][256 bytes] with the 16-byte chunk index
+// XOR-ed with (row & 7), so that the eight row addresses of an ldmatrix hit
+// eight different bank groups.
 // The softmax weights are the fp32 accumulators of S; they enter the second
 // contraction as a 16-bit value plus a 16-bit residual (two mma passes), so
 // the result keeps fp32-level accuracy instead of the 2^-9 of a bf16 weight.
@@ -63,30 +69,64 @@ __device__ __forceinline__ void mma_16816<__half>(float (&d)[4], uint32_t a0, ui
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
 }
 
-__device__ __forceinline__ uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t r;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-  return r;
-}
-
 constexpr int kGqaRows = 16;            // rows per warp per iteration
 constexpr int kGqaHeads = 16;           // M of the mma: most query heads one block serves
 constexpr int kGqaPad = 4;              // floats of padding per head row of the block-level combine
 
-// kHi: more than 8 query heads per K/V head (rows 8..15 of the M dimension are live).
-template <typename T, int kMode, bool kHi, bool kAligned32>
-__global__ void __launch_bounds__(kThreads, kHi ? 2 : 3)
+constexpr int kStagedDepth = 3;                          // tiles per warp in the ring
+constexpr int kStagedTileBytes = kGqaRows * 256;         // one tensor's tile
+constexpr int kStagedWarpBytes = kStagedDepth * 2 * kStagedTileBytes;
+constexpr int kStagedSmemBytes = kWarps * kStagedWarpBytes;   // 96 KB: two blocks per SM
+// A chunk is worked through in windows: the block's warps meet at every window's end (and, for lists, stage
+// the next window's positions).  Meeting often keeps the four warps on neighbouring rows, which the memory
+// system rewards (full context at 32 query heads over 8 / 4 / 2 K/V heads: 6.9 / 6.3 / 5.4 TB/s with windows
+// of 256 rows, 6.7 / 6.2 / 5.4 with 512, 6.5 / 6.0 / 5.4 with 1024, 6.3 / 5.8 / 5.2 without windows), but each
+// meeting lets the ring run empty once (windows of 64 rows: 5.7 / 5.2 / 4.6 TB/s).
+constexpr int kStagedWindow = 512;                       // list entries staged at a time
+constexpr int kStagedDenseWindow = 256;                  // full context: rows between two meetings of the warps
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// 16-byte asynchronous copy global -> shared, not kept in L1, evict-first in L2; src_bytes = 0 writes zeros.
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes, uint64_t policy) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;"
+               ::"r"(dst), "l"(src), "r"(src_bytes), "l"(policy)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+
+// byte offset of 16-byte chunk `chunk` of row `row` inside a swizzled [16][256 B] tile
+__device__ __forceinline__ uint32_t tile_offset(int row, int chunk) {
+  return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4));
+}
+
+template <typename T, int kMode, bool kHi>
+__global__ void __launch_bounds__(kThreads, 2)
 decode_partial_gqa_kernel(const DecodeParams p) {
   constexpr int D = 128;
   constexpr bool kSparse = kMode != kDense;
   constexpr int kLiveHeads = kHi ? 16 : 8;
   static_assert(kMode == kDense || kMode == kIndex || kMode == kSpans,
                 "blocked lists take the one-head-per-block kernel");
+  static_assert(kWarps * kLiveHeads * (D + kGqaPad) * 4 <= kStagedSmemBytes, "the combine reuses the ring");
 
-  __shared__ int32_t s_idx[kSparse ? kMaxChunk : 1];
-  __shared__ __align__(16) float s_acc[kWarps][kLiveHeads][D + kGqaPad];
+  extern __shared__ __align__(128) unsigned char s_ring[];
+  __shared__ int32_t s_idx[kSparse ? kStagedWindow : 1];
+  __shared__ __align__(128) unsigned char s_qtile[kGqaHeads * 256];   // Q of the group, swizzled like a row tile
   __shared__ float s_m[kWarps][kLiveHeads], s_l[kWarps][kLiveHeads];
-  __shared__ uint32_t s_q[kHi ? 32 : 16][32];         // query fragments, [word][lane]: the same for every warp
   __shared__ typename std::conditional<kMode == kSpans, SpanRuns, int>::type s_runs;
 
   const int chunk_id = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
@@ -102,7 +142,6 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   int n, c;
   request_sizes(p, b, n, c, flags);
   if constexpr (kMode == kSpans) {
-    // the request's spans -> disjoint ascending runs in shared memory
     const int first = p.span_offsets ? __ldg(p.span_offsets + b) : b * p.span_cap;
     const int S = p.span_offsets ? __ldg(p.span_offsets + b + 1) - first : p.span_cap;
     const int total = merge_spans_block<kThreads>(s_runs, p.spans + first, S, p.span_cap, n);
@@ -117,10 +156,8 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   if (start >= c && chunk_id > 0) return;
   const int cnt = max(0, min(p.chunk, c - start));
 
-  // A block may own more list entries than the staging area holds: it works through them in windows of
-  // kMaxChunk entries (checked, translated for a paged cache, staged, consumed).
   auto stage_window = [&](int w0, int wn) {
-    if constexpr (kMode == kSpans) {                  // positions by arithmetic on the runs
+    if constexpr (kMode == kSpans) {
       int32_t* out = (kvh == 0 && p.index_out) ? p.index_out + (int64_t)b * p.index_stride + start + w0 : nullptr;
       for (int i = tid; i < wn; i += kThreads) {
         const int v = span_position(s_runs, start + w0 + i);
@@ -142,171 +179,178 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       s_idx[i] = v;
     }
   };
-  if (kSparse) stage_window(0, min(cnt, kMaxChunk));
-  // query fragments: dims [32j, 32j+32) of heads g and g+8 of this K/V head.  They are the same for all
-  // warps and live in shared memory: sixteen registers per lane are worth a third block per SM here.
-  if (warp == 0) {
-    const T* q0 = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)(kvh * G) * p.q_sh + 32 * j;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint4 a = make_uint4(0u, 0u, 0u, 0u), h8 = make_uint4(0u, 0u, 0u, 0u);
-      if (g < G) a = ld_stream_16B(q0 + (int64_t)g * p.q_sh + 8 * i);
-      if (kHi && g + 8 < G) h8 = ld_stream_16B(q0 + (int64_t)(g + 8) * p.q_sh + 8 * i);
-      s_q[4 * i][lane] = a.x; s_q[4 * i + 1][lane] = a.y; s_q[4 * i + 2][lane] = a.z; s_q[4 * i + 3][lane] = a.w;
-      if (kHi) {
-        s_q[16 + 4 * i][lane] = h8.x; s_q[16 + 4 * i + 1][lane] = h8.y;
-        s_q[16 + 4 * i + 2][lane] = h8.z; s_q[16 + 4 * i + 3][lane] = h8.w;
-      }
+  if (kSparse) stage_window(0, min(cnt, kStagedWindow));
+  // the group's query rows -> shared memory (rows of heads that do not exist are zero)
+  {
+    const int row = tid >> 3, c0 = (tid & 7) * 2;
+    uint4 a = make_uint4(0u, 0u, 0u, 0u), c2 = make_uint4(0u, 0u, 0u, 0u);
+    if (row < G) {
+      const T* src = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)(kvh * G + row) * p.q_sh + 8 * c0;
+      a = ld_stream_16B(src);
+      c2 = ld_stream_16B(src + 8);
     }
+    *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0)) = a;
+    *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0 + 1)) = c2;
   }
   __syncthreads();
+  // A fragments of Q for the eight k-steps: registers for the whole block's life
+  uint32_t qa[8][4];
+  {
+    const int m = lane >> 3, r = lane & 7;
+    const uint32_t base = smem_u32(s_qtile);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) ldmatrix_x4(qa[ks], base + tile_offset((m & 1) * 8 + r, 2 * ks + (m >> 1)));
+  }
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
   const char* kbase = reinterpret_cast<const char*>(
-      reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)kvh * p.k_sh + 32 * j);
+      reinterpret_cast<const T*>(p.k) + (int64_t)b * p.k_sb + (int64_t)kvh * p.k_sh);
   const char* vbase = reinterpret_cast<const char*>(
-      reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)kvh * p.v_sh + 16 * g);
+      reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)kvh * p.v_sh);
+  const uint32_t ring = smem_u32(s_ring) + warp * kStagedWarpBytes;
 
-  // running softmax state of heads g (lo) and g+8 (hi); sums are per lane until the end
+  // running softmax state of heads g (lo) and g+8 (hi); sums are per lane until the end.
+  // o[nt][e]: dims 8 nt + 2j + (e & 1) of head g (e < 2) or g + 8 (e >= 2)
   float m_lo = neg_inf(), m_hi = neg_inf(), l_lo = 0.f, l_hi = 0.f;
   float o[16][4];
 #pragma unroll
   for (int u = 0; u < 16; ++u) { o[u][0] = 0.f; o[u][1] = 0.f; o[u][2] = 0.f; o[u][3] = 0.f; }
 
-  for (int w0 = 0; w0 < cnt; w0 += kMaxChunk) {
-  const int wn = min(kMaxChunk, cnt - w0);
-  if (kSparse && w0 > 0) {
-    __syncthreads();                                   // every warp is done with the previous window
-    stage_window(w0, wn);
-    __syncthreads();
-  }
-  for (int t = warp * kGqaRows; t < wn; t += kWarps * kGqaRows) {
-    // which of the tile's 16 rows exist (lane r and r+16 both answer for row r)
-    int my_pos = -1;
-    {
-      const int r = t + (lane & 15);
-      if (r < wn) my_pos = kSparse ? s_idx[r] : start + w0 + r;
+  constexpr int kWindow = kSparse ? kStagedWindow : kStagedDenseWindow;
+  for (int w0 = 0; w0 < cnt; w0 += kWindow) {
+    const int wn = min(kWindow, cnt - w0);
+    if (kSparse && w0 > 0) {
+      __syncthreads();                                 // every warp is done with the previous window
+      stage_window(w0, wn);
+      __syncthreads();
     }
-    const uint32_t live = __ballot_sync(0xffffffffu, my_pos >= 0) & 0xffffu;
-    auto row_pos = [&](int r) { return __shfl_sync(0xffffffffu, my_pos, r); };
-
-    // K: row g of each half (64 bytes per lane per row); V: rows 2j, 2j+1, 2j+8, 2j+9 (32 bytes each)
-    uint32_t kf[2][16], vf[4][8];
+    const int first_row = warp * kGqaRows;
+    const int nk = wn > first_row ? (wn - first_row + kWarps * kGqaRows - 1) / (kWarps * kGqaRows) : 0;
+    // position of row (lane & 15) of this warp's k-th tile, -1 if there is none
+    auto tile_pos = [&](int k) {
+      const int r = first_row + k * (kWarps * kGqaRows) + (lane & 15);
+      return r < wn ? (kSparse ? s_idx[r] : start + w0 + r) : -1;
+    };
+    // requests tile k of the window (if it exists) into slot k % depth; always closes a copy group
+    auto request = [&](int k) {
+      if (k < nk) {
+        const int my_pos = tile_pos(k);
+        const uint32_t slot = ring + (uint32_t)(k % kStagedDepth) * (2 * kStagedTileBytes);
+        const int chunk = lane & 15;
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      const int pos = row_pos(nt * 8 + g);
-      if (pos >= 0) {
-        const char* src = kbase + (uint64_t)(uint32_t)pos * p.k_row_bytes;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {                 // whole 32-byte sectors per request
-          Piece pc;
-          load_piece<kAligned32>(pc, src + 32 * i);
-#pragma unroll
-          for (int w = 0; w < 8; ++w) kf[nt][8 * i + w] = pc.w[w];
+        for (int i = 0; i < 8; ++i) {
+          const int r = 2 * i + (lane >> 4);
+          const int pos = __shfl_sync(0xffffffffu, my_pos, r);
+          const uint32_t bytes = pos >= 0 ? 16u : 0u;
+          const uint64_t row = pos >= 0 ? (uint64_t)(uint32_t)pos : 0ull;
+          const uint32_t off = tile_offset(r, chunk);
+          cp_async_16(slot + off, kbase + row * p.k_row_bytes + chunk * 16, bytes, policy);
+          cp_async_16(slot + kStagedTileBytes + off, vbase + row * p.v_row_bytes + chunk * 16, bytes, policy);
         }
-      } else {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) kf[nt][i] = 0u;
       }
-    }
+      cp_async_commit();
+    };
 #pragma unroll
-    for (int rr = 0; rr < 4; ++rr) {
-      const int pos = row_pos(2 * j + (rr & 1) + 8 * (rr >> 1));
-      if (pos >= 0) {
-        const char* src = vbase + (uint64_t)(uint32_t)pos * p.v_row_bytes;
-        Piece pc;
-        load_piece<kAligned32>(pc, src);
-#pragma unroll
-        for (int w = 0; w < 8; ++w) vf[rr][w] = pc.w[w];
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) vf[rr][i] = 0u;          // weight 0 times anything stored there must stay 0
-      }
-    }
+    for (int k = 0; k < kStagedDepth - 1; ++k) request(k);
+    for (int k = 0; k < nk; ++k) {
+      __syncwarp();                                    // the slot about to be refilled has been read by every lane
+      request(k + kStagedDepth - 1);
+      cp_async_wait<kStagedDepth - 1>();               // tile k has landed (for this lane's copies) ...
+      __syncwarp();                                    // ... and for every other lane's
+      const uint32_t live = __ballot_sync(0xffffffffu, tile_pos(k) >= 0) & 0xffffu;
+      if (live == 0u) continue;                        // warp-uniform: nothing to add
+      const uint32_t kt = ring + (uint32_t)(k % kStagedDepth) * (2 * kStagedTileBytes), vt = kt + kStagedTileBytes;
+      const int mm = lane >> 3, rr = lane & 7;
 
-    // S = Q . K^T for the two 8-row halves
-    float s[2][4];
+      // S = Q . K^T: two n-tiles of 8 rows
+      float s[2][4];
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f;
+      for (int nt = 0; nt < 2; ++nt) { s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f; }
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        mma_16816<T>(s[nt], s_q[2 * ks][lane], kHi ? s_q[16 + 2 * ks][lane] : 0u, s_q[2 * ks + 1][lane],
-                     kHi ? s_q[16 + 2 * ks + 1][lane] : 0u, kf[nt][2 * ks], kf[nt][2 * ks + 1], s[nt]);
-    }
-    // lane (g, j) now holds, for heads g (s[.][0..1]) and g+8 (s[.][2..3]), the rows nt*8 + 2j + {0, 1}
-    float mt_lo = neg_inf(), mt_hi = neg_inf();
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const bool ok = (live >> (nt * 8 + 2 * j + e)) & 1u;
-        s[nt][e] = ok ? s[nt][e] * p.scale_log2 : neg_inf();
-        s[nt][2 + e] = ok ? s[nt][2 + e] * p.scale_log2 : neg_inf();
-        mt_lo = fmaxf(mt_lo, s[nt][e]);
-        mt_hi = fmaxf(mt_hi, s[nt][2 + e]);
+      for (int ks = 0; ks < 8; ++ks) {
+        uint32_t kb[4];                                // rows 0-7: k lo, k hi; rows 8-15: k lo, k hi
+        ldmatrix_x4(kb, kt + tile_offset((mm >> 1) * 8 + rr, 2 * ks + (mm & 1)));
+        mma_16816<T>(s[0], qa[ks][0], kHi ? qa[ks][1] : 0u, qa[ks][2], kHi ? qa[ks][3] : 0u, kb[0], kb[1], s[0]);
+        mma_16816<T>(s[1], qa[ks][0], kHi ? qa[ks][1] : 0u, qa[ks][2], kHi ? qa[ks][3] : 0u, kb[2], kb[3], s[1]);
       }
-    mt_lo = fmaxf(mt_lo, __shfl_xor_sync(0xffffffffu, mt_lo, 1));
-    mt_lo = fmaxf(mt_lo, __shfl_xor_sync(0xffffffffu, mt_lo, 2));
-    if (kHi) {
-      mt_hi = fmaxf(mt_hi, __shfl_xor_sync(0xffffffffu, mt_hi, 1));
-      mt_hi = fmaxf(mt_hi, __shfl_xor_sync(0xffffffffu, mt_hi, 2));
-    }
-    if (live == 0u) continue;                          // warp-uniform: nothing to add
-    const float mn_lo = fmaxf(m_lo, mt_lo), mn_hi = fmaxf(m_hi, mt_hi);
-    if (mn_lo > m_lo) {
-      const float alpha = fast_exp2(m_lo - mn_lo);
-      l_lo *= alpha;
+      // lane (g, j) holds, for heads g (s[.][0..1]) and g+8 (s[.][2..3]), the rows nt*8 + 2j + {0, 1}
+      float mt_lo = neg_inf(), mt_hi = neg_inf();
 #pragma unroll
-      for (int u = 0; u < 16; ++u) { o[u][0] *= alpha; o[u][1] *= alpha; }
-      m_lo = mn_lo;
-    }
-    if (kHi && mn_hi > m_hi) {
-      const float alpha = fast_exp2(m_hi - mn_hi);
-      l_hi *= alpha;
+      for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-      for (int u = 0; u < 16; ++u) { o[u][2] *= alpha; o[u][3] *= alpha; }
-      m_hi = mn_hi;
-    }
-    // weights, split into a 16-bit value and a 16-bit residual; A fragments of P[16 heads, 16 rows]
-    uint32_t pa[4], pr[4];
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      const float w0 = fast_exp2(s[nt][0] - m_lo), w1 = fast_exp2(s[nt][1] - m_lo);   // -inf gives 0
-      l_lo += w0 + w1;
-      pa[2 * nt] = pack2<T>(w0, w1);
-      const float2 back = unpack2<T>(pa[2 * nt]);
-      pr[2 * nt] = pack2<T>(w0 - back.x, w1 - back.y);
+        for (int e = 0; e < 2; ++e) {
+          const bool ok = (live >> (nt * 8 + 2 * j + e)) & 1u;
+          s[nt][e] = ok ? s[nt][e] * p.scale_log2 : neg_inf();
+          s[nt][2 + e] = ok ? s[nt][2 + e] * p.scale_log2 : neg_inf();
+          mt_lo = fmaxf(mt_lo, s[nt][e]);
+          mt_hi = fmaxf(mt_hi, s[nt][2 + e]);
+        }
+      mt_lo = fmaxf(mt_lo, __shfl_xor_sync(0xffffffffu, mt_lo, 1));
+      mt_lo = fmaxf(mt_lo, __shfl_xor_sync(0xffffffffu, mt_lo, 2));
       if (kHi) {
-        const float x0 = fast_exp2(s[nt][2] - m_hi), x1 = fast_exp2(s[nt][3] - m_hi);
-        l_hi += x0 + x1;
-        pa[2 * nt + 1] = pack2<T>(x0, x1);
-        const float2 bk = unpack2<T>(pa[2 * nt + 1]);
-        pr[2 * nt + 1] = pack2<T>(x0 - bk.x, x1 - bk.y);
-      } else {
-        pa[2 * nt + 1] = 0u;
-        pr[2 * nt + 1] = 0u;
+        mt_hi = fmaxf(mt_hi, __shfl_xor_sync(0xffffffffu, mt_hi, 1));
+        mt_hi = fmaxf(mt_hi, __shfl_xor_sync(0xffffffffu, mt_hi, 2));
       }
-    }
-    // O += P . V, one n-tile (8 of this lane group's dims) at a time
+      const float mn_lo = fmaxf(m_lo, mt_lo), mn_hi = fmaxf(m_hi, mt_hi);
+      if (mn_lo > m_lo) {
+        const float alpha = fast_exp2(m_lo - mn_lo);
+        l_lo *= alpha;
 #pragma unroll
-    for (int u = 0; u < 16; ++u) {
-      const uint32_t sel = (u & 1) ? 0x7632u : 0x5410u;
-      const uint32_t b0 = byte_perm(vf[0][u >> 1], vf[1][u >> 1], sel);
-      const uint32_t b1 = byte_perm(vf[2][u >> 1], vf[3][u >> 1], sel);
-      if (kHi) {
-        mma_16816<T>(o[u], pa[0], pa[1], pa[2], pa[3], b0, b1, o[u]);
-        mma_16816<T>(o[u], pr[0], pr[1], pr[2], pr[3], b0, b1, o[u]);
-      } else {
-        // rows 8..15 of the M dimension are unused: feed zeros, drop what comes back
-        float acc[4] = {o[u][0], o[u][1], 0.f, 0.f};
-        mma_16816<T>(acc, pa[0], 0u, pa[2], 0u, b0, b1, acc);
-        mma_16816<T>(acc, pr[0], 0u, pr[2], 0u, b0, b1, acc);
-        o[u][0] = acc[0];
-        o[u][1] = acc[1];
+        for (int u = 0; u < 16; ++u) { o[u][0] *= alpha; o[u][1] *= alpha; }
+        m_lo = mn_lo;
+      }
+      if (kHi && mn_hi > m_hi) {
+        const float alpha = fast_exp2(m_hi - mn_hi);
+        l_hi *= alpha;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) { o[u][2] *= alpha; o[u][3] *= alpha; }
+        m_hi = mn_hi;
+      }
+      // weights, split into a 16-bit value and a 16-bit residual: A fragments of P[16 heads, 16 rows]
+      // (a0: head g, rows 2j..; a1: head g+8, rows 2j..; a2: head g, rows 8+2j..; a3: head g+8, rows 8+2j..)
+      uint32_t pa[4], pr[4];
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const float w0 = fast_exp2(s[nt][0] - m_lo), w1 = fast_exp2(s[nt][1] - m_lo);   // -inf gives 0
+        l_lo += w0 + w1;
+        pa[2 * nt] = pack2<T>(w0, w1);
+        const float2 back = unpack2<T>(pa[2 * nt]);
+        pr[2 * nt] = pack2<T>(w0 - back.x, w1 - back.y);
+        if (kHi) {
+          const float x0 = fast_exp2(s[nt][2] - m_hi), x1 = fast_exp2(s[nt][3] - m_hi);
+          l_hi += x0 + x1;
+          pa[2 * nt + 1] = pack2<T>(x0, x1);
+          const float2 bk = unpack2<T>(pa[2 * nt + 1]);
+          pr[2 * nt + 1] = pack2<T>(x0 - bk.x, x1 - bk.y);
+        } else {
+          pa[2 * nt + 1] = 0u;
+          pr[2 * nt + 1] = 0u;
+        }
+      }
+      // O += P . V, sixteen dims (two n-tiles) per ldmatrix
+#pragma unroll
+      for (int dn = 0; dn < 8; ++dn) {
+        uint32_t vb[4];                                // dims 16dn..+7: rows 0-7, rows 8-15; dims 16dn+8..+15: the same
+        ldmatrix_x4_trans(vb, vt + tile_offset((mm & 1) * 8 + rr, 2 * dn + (mm >> 1)));
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int u = 2 * dn + half;
+          if (kHi) {
+            mma_16816<T>(o[u], pa[0], pa[1], pa[2], pa[3], vb[2 * half], vb[2 * half + 1], o[u]);
+            mma_16816<T>(o[u], pr[0], pr[1], pr[2], pr[3], vb[2 * half], vb[2 * half + 1], o[u]);
+          } else {
+            // rows 8..15 of the M dimension are unused: feed zeros, drop what comes back
+            float acc[4] = {o[u][0], o[u][1], 0.f, 0.f};
+            mma_16816<T>(acc, pa[0], 0u, pa[2], 0u, vb[2 * half], vb[2 * half + 1], acc);
+            mma_16816<T>(acc, pr[0], 0u, pr[2], 0u, vb[2 * half], vb[2 * half + 1], acc);
+            o[u][0] = acc[0];
+            o[u][1] = acc[1];
+          }
+        }
       }
     }
+    cp_async_wait<0>();                                // only empty groups can be pending here
   }
-
-  }                                                    // windows
   if (p.dev_status && kvh == 0) {
     const uint32_t f = (tid == 0 && chunk_id == 0) ? flags : (flags & SSA_DEV_BAD_INDEX);
     if (f) atomicOr(p.dev_status, f);
@@ -314,7 +358,9 @@ decode_partial_gqa_kernel(const DecodeParams p) {
 
   if (!p.early_release) grid_launch_dependents();
 
-  // per-warp triples -> shared memory.  o[u][e] of lane (g, j) is dim 32j + 16e + u of head g (+8 for e+2).
+  // per-warp triples -> shared memory (the ring is free now)
+  __syncthreads();
+  float (*s_acc)[kLiveHeads][D + kGqaPad] = reinterpret_cast<float (*)[kLiveHeads][D + kGqaPad]>(s_ring);
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   if (kHi) {
@@ -323,12 +369,8 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   }
 #pragma unroll
   for (int u = 0; u < 16; ++u) {
-    s_acc[warp][g][32 * j + u] = o[u][0];
-    s_acc[warp][g][32 * j + 16 + u] = o[u][1];
-    if (kHi) {
-      s_acc[warp][g + 8][32 * j + u] = o[u][2];
-      s_acc[warp][g + 8][32 * j + 16 + u] = o[u][3];
-    }
+    *reinterpret_cast<float2*>(&s_acc[warp][g][8 * u + 2 * j]) = make_float2(o[u][0], o[u][1]);
+    if (kHi) *reinterpret_cast<float2*>(&s_acc[warp][g + 8][8 * u + 2 * j]) = make_float2(o[u][2], o[u][3]);
   }
   if (j == 0) {
     s_m[warp][g] = m_lo; s_l[warp][g] = l_lo;
