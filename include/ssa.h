@@ -463,7 +463,7 @@ int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, cons
  *   neither               the library decides: one kernel when max_spans <= 32,
  *                         the workspace suffices, the inputs are not fetched by
  *                         kernel (that fetch is fused with the index launch)
- *                         and the attention grid is at most four waves of
+ *                         and the attention grid is at most three waves of
  *                         thread blocks - where every block repeating the merge
  *                         of its request's spans costs less than a launch.
  * Errors: SSA_ERR_NULL for a NULL desc/step or an inconsistent copy request,

@@ -688,14 +688,14 @@ int32_t one_kernel_span_limit() { return kDirectSpans; }
 
 // Every block of the span-list kernel repeats the merge of its request's spans (about a microsecond per wave
 // of blocks when a warp can do it alone), the index kernel does it once per request but costs a launch of its
-// own (3-4 us exposed).  Measured on the five workloads: one kernel wins or ties up to about four waves.
+// own (about 3 us exposed): one kernel up to three waves of blocks.
 bool one_kernel_step_pays(const ssa_attn_desc* d, int32_t max_selected, int32_t max_spans, size_t ws_bytes) {
   Plan pl;
   if (max_spans <= 0 || max_spans > 32 || !d || check_desc(d) != SSA_OK || !make_plan(d, max_selected, &pl))
     return false;
   if (ws_bytes < pl.total_bytes + counts_bytes(d)) return false;
   const long long units = shares_rows(d) ? (long long)d->B * d->H_kv : (long long)d->B * d->H;
-  return units * pl.n_chunks <= 4ll * SSA_MIN_BLOCKS * sm_count();
+  return units * pl.n_chunks <= 3ll * SSA_MIN_BLOCKS * sm_count();
 }
 
 // Scratch of ssa_decode_attn_sparse_noalloc: part of the library's device image.
