@@ -40,6 +40,8 @@ What is stated here, and where the paper defines it:
 * ``decode_attn_sparse_multiq``  several query rows per head over one
                           selected set (outside the paper, which decodes one
                           token per step): the set form applied row by row.
+* ``decode_e4m3``         the 8-bit cache storage format (outside the paper),
+                          from the format's definition.
 * ``merge_partials``      recombination of (max, sum, accumulator) partial
                           results of disjoint subsets; not in the paper (its
                           kernel runs one thread block per head and request),
@@ -85,7 +87,10 @@ def decode_bits(u16, dtype: str) -> np.ndarray:
 
     ``bf16``: the pattern is the upper half of an IEEE binary32.
     ``f16`` : IEEE binary16.
+    ``e4m3``: 8-bit patterns (uint8), see ``decode_e4m3``.
     """
+    if dtype == "e4m3":
+        return decode_e4m3(u16)
     a = np.ascontiguousarray(u16)
     if a.dtype != np.uint16:
         raise TypeError("expected uint16 bit patterns")
@@ -95,6 +100,25 @@ def decode_bits(u16, dtype: str) -> np.ndarray:
     if dtype == "f16":
         return a.view(np.float16).astype(np.float64)
     raise ValueError(f"unknown storage dtype {dtype!r}")
+
+
+def decode_e4m3(u8) -> np.ndarray:
+    """Exact value of 8-bit "e4m3" storage patterns (1 sign bit, 4 exponent
+    bits with bias 7, 3 mantissa bits; the format has no infinities and its
+    only NaN is exponent 15 with mantissa 7) as float64, written out from the
+    format's definition bit field by bit field:
+      exponent 0      : (mantissa / 8) * 2^-6           (subnormal, and zero)
+      otherwise       : (1 + mantissa / 8) * 2^(exponent - 7), up to 448.
+    The paper stores the cache in 16 bits; 8-bit storage is outside it."""
+    a = np.ascontiguousarray(u8)
+    if a.dtype != np.uint8:
+        raise TypeError("expected uint8 bit patterns")
+    sign = np.where(a >> 7, -1.0, 1.0)
+    e = ((a >> 3) & 0xF).astype(np.int64)
+    m = (a & 0x7).astype(np.float64)
+    val = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    val = np.where((e == 15) & ((a & 0x7) == 7), np.nan, val)
+    return sign * val
 
 
 # --------------------------------------------------------------------------
@@ -357,9 +381,13 @@ def merge_partials(ms, ls, accs):
 # batch forms over a KV cache (logical layout [B, H, T, D])
 # --------------------------------------------------------------------------
 def _as_f64(a, dtype):
+    """dtype may name two storage types, "query/cache" (e.g. "bf16/e4m3": 16-bit
+    queries over an 8-bit cache); uint8 arrays are always e4m3 patterns."""
     a = np.asarray(a)
+    if a.dtype == np.uint8:
+        return decode_e4m3(a)
     if a.dtype == np.uint16:
-        return decode_bits(a, dtype)
+        return decode_bits(a, dtype.split("/")[0])
     return a.astype(np.float64)
 
 
