@@ -585,6 +585,46 @@ def variants_outside_the_paper(torch, ssa, timer, n_iter=100):
                      "kv_gbs_sparse": round(sel / ts / 1e3), "kv_gbs_dense": round(B * T * 2 * hkv * D * 2 / td / 1e3)})
         del ds
         torch.cuda.empty_cache()
+    # 8-bit (e4m3) cache storage against the 16-bit cache: same shapes and lists (cfg 5 at 10 %, multi-head)
+    wl = inputs.make_config(5, density=0.10)
+    ncopy = 3
+    ds = DecodeStep(wl, kv_copies=ncopy)
+    ds.build_index()
+    torch.cuda.synchronize()
+    rows_sel, rows_all = int(ds.counts.sum().item()), wl.B * wl.max_ctx
+    k8 = [k.to(torch.float8_e4m3fn) for k in ds.k_store]
+    v8 = [v.to(torch.float8_e4m3fn) for v in ds.v_store]
+    desc8 = ssa.make_desc(ds.q, k8[0], v8[0], ds.out, max_ctx=wl.max_ctx)
+
+    def sparse8(i):
+        ssa.decode_attn_sparse(desc8, ds.q, k8[i % ncopy], v8[i % ncopy], ds.ctx_lens, ds.index, ds.counts,
+                               ds.max_selected, ds.out, ds.lse, ds.workspace, ds.status)
+
+    def dense8(i):
+        ssa.decode_attn_dense(desc8, ds.q, k8[i % ncopy], v8[i % ncopy], ds.ctx_lens, ds.out, ds.lse, ds.workspace,
+                              ds.status)
+
+    def sparse16(i):
+        ds.select_copy(i % ncopy)
+        ds.attend_sparse()
+
+    def dense16(i):
+        ds.select_copy(i % ncopy)
+        ds.attend_dense()
+
+    for i in range(3):
+        sparse8(i), dense8(i), sparse16(i), dense16(i)
+    t8s = timer.run(sparse8, n_iter) / n_iter * 1e3
+    t8d = timer.run(dense8, n_iter // 4) / (n_iter // 4) * 1e3
+    t16s = timer.run(sparse16, n_iter) / n_iter * 1e3
+    t16d = timer.run(dense16, n_iter // 4) / (n_iter // 4) * 1e3
+    row8 = 2 * wl.H * wl.D                               # K + V bytes of one position over all heads, one byte each
+    fp8 = {"workload": "cfg5 10%: B=32, 32 heads x 128, ctx 8192; cache stored as e4m3 bytes, bf16 queries",
+           "sparse_attn_us": round(t8s, 2), "dense_us": round(t8d, 2),
+           "kv_gbs_sparse": round(rows_sel * row8 / t8s / 1e3), "kv_gbs_dense": round(rows_all * row8 / t8d / 1e3),
+           "bf16_cache_sparse_attn_us": round(t16s, 2), "bf16_cache_dense_us": round(t16d, 2)}
+    del ds, k8, v8
+    torch.cuda.empty_cache()
     # paged cache: cfg 2 shapes, token-major pool, 16-row pages in shuffled order, against the contiguous call
     wl = inputs.make_config(2)
     ncopy = 4
@@ -620,9 +660,9 @@ def variants_outside_the_paper(torch, ssa, timer, n_iter=100):
     del ds, pools
     torch.cuda.empty_cache()
     return {"what": "outside the paper: grouped query heads (B=32, 32 query heads x 128, ctx 8192, 10% selected; rows "
-                    "of a K/V head are read once for its whole group) and a paged cache (cfg 2 shapes, 16-row pages "
-                    "in shuffled order, attention call alone)",
-            "grouped_heads": rows,
+                    "of a K/V head are read once for its whole group), an 8-bit cache and a paged cache (cfg 2 shapes, "
+                    "16-row pages in shuffled order, attention call alone)",
+            "grouped_heads": rows, "fp8_cache": fp8,
             "paged_cfg2": {"page_size": ps, "paged_attn_us": round(tp, 2), "contiguous_attn_us": round(tc, 2)}}
 
 

@@ -64,7 +64,7 @@ enum {
 
 #define SSA_MAX_SPANS_PER_SEQ 2048
 
-typedef enum { SSA_F16 = 0, SSA_BF16 = 1, SSA_F32 = 2 } ssa_dtype;
+typedef enum { SSA_F16 = 0, SSA_BF16 = 1, SSA_F32 = 2, SSA_FP8_E4M3 = 3 } ssa_dtype;
 
 /*
  * Geometry of q, the KV cache and the output.  Strides are in ELEMENTS; the
@@ -82,6 +82,13 @@ typedef enum { SSA_F16 = 0, SSA_BF16 = 1, SSA_F32 = 2 } ssa_dtype;
  * query head h reads K/V head h / (H/H_kv); the cache then has H_kv heads).
  * Every base pointer and every stride * element size
  * must be a multiple of 16 bytes.
+ * kv_dtype SSA_FP8_E4M3 (not in the paper, whose cache is 16-bit): K and V are
+ * stored as 8-bit e4m3 values (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
+ * infinities), one byte per element, read as they are - a caller that keeps a
+ * scale with the cache folds K's into `scale` and applies V's to the output;
+ * q is then BF16 and out_dtype BF16 or F32.  Such a cache halves the bytes per
+ * selected row; grouped query heads over it are served one head per thread
+ * block (each head re-reads the rows, mostly from L2).
  */
 typedef struct {
   int32_t B, H, H_kv, D;

@@ -106,16 +106,21 @@ __device__ __forceinline__ void store_out(const DecodeParams& p, int b, int h, i
   else reinterpret_cast<T*>(p.out)[o] = from_float<T>(val);
 }
 
-// 32 bytes of a cache row: eight packed pairs of 16-bit values.
+// A lane's piece of a cache row: 16 values as eight pairs.  16-bit storage: 32 bytes, a pair per word; 8-bit
+// storage: 16 bytes in w[0..3], two pairs per word.
 struct Piece { uint32_t w[8]; };
 
 // A cache row is used once per launch, so the 256-bit loads mark its lines evict-first in L2 as well: they then
 // do not push out what is re-read (index lists, query rows, partial results).  Measured: 4-5 % off every workload
 // (cfg 2 attention 32.4 -> 30.7 us, full context at cfg 2 105 -> 100.5 us); prefetch-size hints on top: nothing.
 // (The qualifier exists for 256-bit loads only, so the 128-bit fallback keeps the default L2 policy.)
-template <bool kAligned32>
+template <bool kAligned32, bool kFp8 = false>
 __device__ __forceinline__ void load_piece(Piece& r, const char* p) {
-  if (kAligned32) {
+  if (kFp8) {
+    const uint4 a = ld_stream_16B(p);
+    r.w[0] = a.x; r.w[1] = a.y; r.w[2] = a.z; r.w[3] = a.w;
+    r.w[4] = 0u; r.w[5] = 0u; r.w[6] = 0u; r.w[7] = 0u;
+  } else if (kAligned32) {
     asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]),
                    "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
@@ -125,6 +130,13 @@ __device__ __forceinline__ void load_piece(Piece& r, const char* p) {
     r.w[0] = a.x; r.w[1] = a.y; r.w[2] = a.z; r.w[3] = a.w;
     r.w[4] = b.x; r.w[5] = b.y; r.w[6] = b.z; r.w[7] = b.w;
   }
+}
+
+// Pair i (0..7) of a piece as two floats.
+template <typename T>
+__device__ __forceinline__ float2 piece_pair(const Piece& r, int i) {
+  if constexpr (kIsFp8<T>) return e4m3x2_to_float2(r.w[i >> 1] >> ((i & 1) * 16));
+  else return unpack2<T>(r.w[i]);
 }
 
 __device__ __forceinline__ void zero_piece(Piece& r) {
@@ -138,6 +150,8 @@ template <typename T, int D, int kMode, bool kAligned32, bool kPaged = false>
 __global__ void __launch_bounds__(kThreads, SSA_MIN_BLOCKS)
 decode_partial_kernel(const DecodeParams p) {
   static_assert(!kPaged || kMode == kIndex, "a paged cache is read through staged positions");
+  using TQ = typename Storage<T>::Query;              // type of the query rows and of a stored output
+  constexpr bool kFp8 = kIsFp8<T>;
   constexpr bool kSparse = kMode != kDense;           // positions come from shared memory
   constexpr int kLanesPerRow = D / 16;                // 32-byte pieces per row
   constexpr int kRowsPerLoad = 32 / kLanesPerRow;     // rows one warp-wide load covers
@@ -183,7 +197,7 @@ decode_partial_kernel(const DecodeParams p) {
   Piece qraw;                                         // re-read by every warp and chunk of the head: plain L2 policy
   {
     const char* qp = reinterpret_cast<const char*>(
-        reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + col * 16);
+        reinterpret_cast<const TQ*>(p.q) + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + col * 16);
     const uint4 a = ld_stream_16B(qp), c4 = ld_stream_16B(qp + 16);
     qraw.w[0] = a.x; qraw.w[1] = a.y; qraw.w[2] = a.z; qraw.w[3] = a.w;
     qraw.w[4] = c4.x; qraw.w[5] = c4.y; qraw.w[6] = c4.z; qraw.w[7] = c4.w;
@@ -310,7 +324,7 @@ decode_partial_kernel(const DecodeParams p) {
   float2 q2[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    q2[i] = unpack2<T>(qraw.w[i]);
+    q2[i] = unpack2<TQ>(qraw.w[i]);
     q2[i].x *= p.scale_log2;
     q2[i].y *= p.scale_log2;
   }
@@ -329,8 +343,8 @@ decode_partial_kernel(const DecodeParams p) {
       for (int u = 0; u < kU; ++u) {
         const int r = t + u * kRowsPerLoad + sub;
         const uint32_t pos = (uint32_t)(kSparse ? s_idx[r] : start + r);
-        load_piece<kAligned32>(kr[u], kbase + (uint64_t)pos * p.k_row_bytes);
-        load_piece<kAligned32>(vr[u], vbase + (uint64_t)pos * p.v_row_bytes);
+        load_piece<kAligned32, kFp8>(kr[u], kbase + (uint64_t)pos * p.k_row_bytes);
+        load_piece<kAligned32, kFp8>(vr[u], vbase + (uint64_t)pos * p.v_row_bytes);
       }
     } else {
 #pragma unroll
@@ -339,8 +353,8 @@ decode_partial_kernel(const DecodeParams p) {
         int pos = -1;
         if (r < cnt) pos = kSparse ? s_idx[r] : start + r;
         if (pos >= 0) {
-          load_piece<kAligned32>(kr[u], kbase + (uint64_t)(uint32_t)pos * p.k_row_bytes);
-          load_piece<kAligned32>(vr[u], vbase + (uint64_t)(uint32_t)pos * p.v_row_bytes);
+          load_piece<kAligned32, kFp8>(kr[u], kbase + (uint64_t)(uint32_t)pos * p.k_row_bytes);
+          load_piece<kAligned32, kFp8>(vr[u], vbase + (uint64_t)(uint32_t)pos * p.v_row_bytes);
           s[u] = 0.f;
         } else {
           zero_piece(kr[u]);
@@ -354,7 +368,7 @@ decode_partial_kernel(const DecodeParams p) {
     for (int u = 0; u < kU; ++u) {
       float2 d2 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) d2 = fma2(q2[i], unpack2<T>(kr[u].w[i]), d2);
+      for (int i = 0; i < 8; ++i) d2 = fma2(q2[i], piece_pair<T>(kr[u], i), d2);
       float d = d2.x + d2.y;
 #pragma unroll
       for (int o = kLanesPerRow / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
@@ -376,7 +390,7 @@ decode_partial_kernel(const DecodeParams p) {
         l += pw;
         const float2 pw2 = make_float2(pw, pw);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = fma2(pw2, unpack2<T>(vr[u].w[i]), acc[i]);
+        for (int i = 0; i < 8; ++i) acc[i] = fma2(pw2, piece_pair<T>(vr[u], i), acc[i]);
       }
     }
   }
@@ -405,7 +419,7 @@ decode_partial_kernel(const DecodeParams p) {
       A = fmaf(s_acc[i][tid], w, A);
     }
     if (p.n_chunks == 1) {
-      store_out<T>(p, b, h, tid, L > 0.f ? A / L : 0.f);
+      store_out<TQ>(p, b, h, tid, L > 0.f ? A / L : 0.f);
       if (tid == 0 && p.lse) p.lse[(int64_t)b * p.H + h] = L > 0.f ? (M + log2f(L)) * kLn2 : neg_inf();
     } else {
       const int64_t slot = ((int64_t)b * p.H + h) * p.n_chunks + chunk_id;
@@ -453,7 +467,7 @@ struct Plan { int chunk, n_chunks; size_t acc_bytes, total_bytes; };
 // Grouped query heads go to the kernel that reads a K/V row once for the whole group.
 static bool shares_rows(const ssa_attn_desc* d) {
   const int group = d->H_kv > 0 ? d->H / d->H_kv : 1;
-  return d->D == 128 && group >= 2 && group <= kGqaHeads;
+  return d->D == 128 && group >= 2 && group <= kGqaHeads && d->kv_dtype != SSA_FP8_E4M3;   // mma takes 16-bit rows
 }
 
 static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
@@ -507,13 +521,19 @@ static int32_t check_desc(const ssa_attn_desc* d) {
   if (d->B <= 0 || d->H <= 0 || d->max_ctx <= 0 || d->B > 65535 || d->H > 65535) return SSA_ERR_SHAPE;
   if (d->D != 64 && d->D != 128) return SSA_ERR_UNSUPPORTED;
   if (d->H_kv <= 0 || d->H % d->H_kv != 0) return SSA_ERR_UNSUPPORTED;
-  if (d->kv_dtype != SSA_F16 && d->kv_dtype != SSA_BF16) return SSA_ERR_DTYPE;
-  if (d->out_dtype != d->kv_dtype && d->out_dtype != SSA_F32) return SSA_ERR_DTYPE;
-  const int64_t strides[] = {d->q_stride_b, d->q_stride_h, d->k_stride_b, d->k_stride_t, d->k_stride_h,
-                             d->v_stride_b, d->v_stride_t, d->v_stride_h, d->o_stride_b, d->o_stride_h};
-  for (int64_t s : strides) {
+  const bool fp8 = d->kv_dtype == SSA_FP8_E4M3;
+  if (d->kv_dtype != SSA_F16 && d->kv_dtype != SSA_BF16 && !fp8) return SSA_ERR_DTYPE;
+  const int32_t q_dtype = fp8 ? SSA_BF16 : d->kv_dtype;            // queries over an 8-bit cache are bf16
+  if (d->out_dtype != q_dtype && d->out_dtype != SSA_F32) return SSA_ERR_DTYPE;
+  const int64_t qo_strides[] = {d->q_stride_b, d->q_stride_h, d->o_stride_b, d->o_stride_h};
+  const int64_t kv_strides[] = {d->k_stride_b, d->k_stride_t, d->k_stride_h, d->v_stride_b, d->v_stride_t, d->v_stride_h};
+  for (int64_t s : qo_strides) {
     if (s < 0) return SSA_ERR_SHAPE;
     if (s % 8 != 0) return SSA_ERR_ALIGN;
+  }
+  for (int64_t s : kv_strides) {                                   // 16 bytes: 8 16-bit or 16 8-bit elements
+    if (s < 0) return SSA_ERR_SHAPE;
+    if (s % (fp8 ? 16 : 8) != 0) return SSA_ERR_ALIGN;
   }
   if (d->k_stride_t >= (1ll << 31) || d->v_stride_t >= (1ll << 31)) return SSA_ERR_SHAPE;
   return SSA_OK;
@@ -525,31 +545,40 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   take_kernel_events(&ev_b, &ev_e);
   dim3 grid((unsigned)p.n_chunks, (unsigned)p.H, (unsigned)B);
   void (*kernel)(const DecodeParams);
-  const bool share = D == 128 && p.kv_group >= 2 && p.kv_group <= kGqaHeads && mode != kBlockMask;
+  using TQ = typename Storage<T>::Query;
+  constexpr bool kFp8 = kIsFp8<T>;
   size_t dynamic_smem = 0;
-  if (share) {
-    grid.y = (unsigned)(p.H / p.kv_group);              // one block per K/V head
-    const bool hi = p.kv_group > 8;
-    if (mode == kIndex)
-      kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true> : decode_partial_gqa_kernel<T, kIndex, false>;
+  bool share = false;
+  if constexpr (!kFp8) {                                // the row-sharing kernel feeds 16-bit rows to the tensor cores
+    share = D == 128 && p.kv_group >= 2 && p.kv_group <= kGqaHeads && mode != kBlockMask;
+    if (share) {
+      grid.y = (unsigned)(p.H / p.kv_group);            // one block per K/V head
+      const bool hi = p.kv_group > 8;
+      if (mode == kIndex)
+        kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true> : decode_partial_gqa_kernel<T, kIndex, false>;
+      else if (mode == kSpans)
+        kernel = hi ? decode_partial_gqa_kernel<T, kSpans, true> : decode_partial_gqa_kernel<T, kSpans, false>;
+      else
+        kernel = hi ? decode_partial_gqa_kernel<T, kDense, true> : decode_partial_gqa_kernel<T, kDense, false>;
+      dynamic_smem = kStagedSmemBytes;
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStagedSmemBytes) != cudaSuccess)
+        return SSA_ERR_CUDA;
+    }
+  }
+  if (!share) {
+    constexpr bool kWide = !kFp8;                       // 8-bit rows are read in 16-byte pieces: one instantiation
+    const bool a32 = kWide && aligned32;
+    if (mode == kIndex && p.page_table)
+      kernel = a32 ? decode_partial_kernel<T, D, kIndex, kWide, true> : decode_partial_kernel<T, D, kIndex, false, true>;
+    else if (mode == kIndex)
+      kernel = a32 ? decode_partial_kernel<T, D, kIndex, kWide> : decode_partial_kernel<T, D, kIndex, false>;
+    else if (mode == kBlockMask)
+      kernel = a32 ? decode_partial_kernel<T, D, kBlockMask, kWide> : decode_partial_kernel<T, D, kBlockMask, false>;
     else if (mode == kSpans)
-      kernel = hi ? decode_partial_gqa_kernel<T, kSpans, true> : decode_partial_gqa_kernel<T, kSpans, false>;
+      kernel = a32 ? decode_partial_kernel<T, D, kSpans, kWide> : decode_partial_kernel<T, D, kSpans, false>;
     else
-      kernel = hi ? decode_partial_gqa_kernel<T, kDense, true> : decode_partial_gqa_kernel<T, kDense, false>;
-    dynamic_smem = kStagedSmemBytes;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStagedSmemBytes) != cudaSuccess)
-      return SSA_ERR_CUDA;
-  } else if (mode == kIndex && p.page_table)
-    kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true, true>
-                       : decode_partial_kernel<T, D, kIndex, false, true>;
-  else if (mode == kIndex)
-    kernel = aligned32 ? decode_partial_kernel<T, D, kIndex, true> : decode_partial_kernel<T, D, kIndex, false>;
-  else if (mode == kBlockMask)
-    kernel = aligned32 ? decode_partial_kernel<T, D, kBlockMask, true> : decode_partial_kernel<T, D, kBlockMask, false>;
-  else if (mode == kSpans)
-    kernel = aligned32 ? decode_partial_kernel<T, D, kSpans, true> : decode_partial_kernel<T, D, kSpans, false>;
-  else
-    kernel = aligned32 ? decode_partial_kernel<T, D, kDense, true> : decode_partial_kernel<T, D, kDense, false>;
+      kernel = a32 ? decode_partial_kernel<T, D, kDense, kWide> : decode_partial_kernel<T, D, kDense, false>;
+  }
   if (ev_b) cudaEventRecord(ev_b, st);
   cudaError_t err = launch_pdl_smem(kernel, grid, dim3(kThreads), dynamic_smem, st, p);
   if (ev_e) cudaEventRecord(ev_e, st);
@@ -558,7 +587,7 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   if (p.n_chunks > 1) {
     DecodeParams pm = p;
     if (mode == kSpans) pm.counts = p.ws_counts;        // the first pass left the list lengths there
-    err = launch_pdl(decode_merge_kernel<T, D>, dim3((unsigned)p.H, (unsigned)B), dim3(D), st, pm);
+    err = launch_pdl(decode_merge_kernel<TQ, D>, dim3((unsigned)p.H, (unsigned)B), dim3(D), st, pm);
     if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
     ++launches;
   }
@@ -659,8 +688,9 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   p.kv_group = d->H / d->H_kv;
   p.k_sb = pg ? 0 : d->k_stride_b; p.k_sh = d->k_stride_h;      // a pool has no batch dimension
   p.v_sb = pg ? 0 : d->v_stride_b; p.v_sh = d->v_stride_h;
-  p.k_row_bytes = (uint32_t)(d->k_stride_t * 2);
-  p.v_row_bytes = (uint32_t)(d->v_stride_t * 2);
+  const int kv_bytes = d->kv_dtype == SSA_FP8_E4M3 ? 1 : 2;
+  p.k_row_bytes = (uint32_t)(d->k_stride_t * kv_bytes);
+  p.v_row_bytes = (uint32_t)(d->v_stride_t * kv_bytes);
   p.o_sb = d->o_stride_b; p.o_sh = d->o_stride_h;
   p.H = d->H; p.max_ctx = d->max_ctx;
   p.index_stride = index_stride; p.max_selected = max_selected;
@@ -678,6 +708,8 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
                    p.k_sb % 16 == 0 && d->k_stride_t % 16 == 0 && d->k_stride_h % 16 == 0 &&
                    p.v_sb % 16 == 0 && d->v_stride_t % 16 == 0 && d->v_stride_h % 16 == 0;
   cudaStream_t st = (cudaStream_t)stream;
+  if (d->kv_dtype == SSA_FP8_E4M3)
+    return d->D == 128 ? launch<Fp8E4M3, 128>(p, d->B, mode, false, st) : launch<Fp8E4M3, 64>(p, d->B, mode, false, st);
   if (d->kv_dtype == SSA_BF16)
     return d->D == 128 ? launch<__nv_bfloat16, 128>(p, d->B, mode, a32, st)
                        : launch<__nv_bfloat16, 64>(p, d->B, mode, a32, st);

@@ -62,6 +62,21 @@ __device__ __forceinline__ uint4 ld_stream_16B(const void* p) {
   return r;
 }
 
+// A K/V cache stored as 8-bit e4m3 values (1 sign, 4 exponent, 3 mantissa bits; outside the paper).  Queries and
+// outputs that go with such a cache are bf16.
+struct Fp8E4M3 { uint8_t bits; };
+template <typename T> struct Storage { using Query = T; };
+template <> struct Storage<Fp8E4M3> { using Query = __nv_bfloat16; };
+template <typename T> constexpr bool kIsFp8 = false;
+template <> constexpr bool kIsFp8<Fp8E4M3> = true;
+
+// Two e4m3 values (the low 16 bits of `pair`) -> two floats (exact: every e4m3 value is an fp16 value).
+__device__ __forceinline__ float2 e4m3x2_to_float2(uint32_t pair) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)pair));
+  return __half22float2(*reinterpret_cast<const __half2*>(&h2));
+}
+
 // Two packed 16-bit storage values -> two floats (exact).
 template <typename T>
 __device__ __forceinline__ float2 unpack2(uint32_t u);

@@ -20,8 +20,8 @@ ERR_NULL, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_CAPACITY, ERR_WORKSPACE, ERR_CUDA
 DEV_BAD_SPAN, DEV_CLIPPED, DEV_OVERFLOW, DEV_BAD_INDEX, DEV_BAD_COUNT, DEV_TOO_MANY_SPANS = 1, 2, 4, 8, 16, 32
 DEV_BAD_REF = 64
 MAX_SPANS_PER_SEQ = 2048
-F16, BF16, F32 = 0, 1, 2
-_DTYPES = {torch.float16: F16, torch.bfloat16: BF16, torch.float32: F32}
+F16, BF16, F32, FP8_E4M3 = 0, 1, 2, 3
+_DTYPES = {torch.float16: F16, torch.bfloat16: BF16, torch.float32: F32, torch.float8_e4m3fn: FP8_E4M3}
 
 
 class AttnDesc(C.Structure):
