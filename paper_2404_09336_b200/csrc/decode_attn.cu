@@ -152,6 +152,7 @@ decode_partial_kernel(const DecodeParams p) {
   static_assert(!kPaged || kMode == kIndex, "a paged cache is read through staged positions");
   using TQ = typename Storage<T>::Query;              // type of the query rows and of a stored output
   constexpr bool kFp8 = kIsFp8<T>;
+  constexpr int kU = kFp8 ? 2 * SSA_U : SSA_U;        // 8-bit pieces are half as large: twice as many in flight
   constexpr bool kSparse = kMode != kDense;           // positions come from shared memory
   constexpr int kLanesPerRow = D / 16;                // 32-byte pieces per row
   constexpr int kRowsPerLoad = 32 / kLanesPerRow;     // rows one warp-wide load covers
