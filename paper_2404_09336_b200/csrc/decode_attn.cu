@@ -430,25 +430,57 @@ decode_partial_kernel(const DecodeParams p) {
   }
 }
 
+// Pass 2.  The kernel is pure latency (a few KB per block), so everything it may need is requested in one go,
+// before the request's list length is known: the (max, sum) pairs of all n_chunks slots and the first eight
+// accumulator rows.  Slots of chunks that do not exist were never written; what is read from them is not used.
+constexpr int kMergeStage = 512;       // (max, sum) pairs staged in shared memory; more chunks: read in place
+constexpr int kMergeAhead = 8;         // accumulator rows requested before the sizes are known
+
 template <typename T, int D>
 __global__ void __launch_bounds__(D)
 decode_merge_kernel(const DecodeParams p) {
+  __shared__ float2 s_ml[kMergeStage];
   const int h = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
   grid_dependency_wait();
   grid_launch_dependents();
+  const int64_t base = ((int64_t)b * p.H + h) * p.n_chunks;
+  const bool staged = p.n_chunks <= kMergeStage;
+  if (staged)
+    for (int k = d; k < p.n_chunks; k += D) s_ml[k] = p.ws_ml[base + k];
+  float ahead[kMergeAhead];
+#pragma unroll
+  for (int k = 0; k < kMergeAhead; ++k) ahead[k] = k < p.n_chunks ? p.ws_acc[(base + k) * D + d] : 0.f;
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
   const int ns = c > 0 ? (c + p.chunk - 1) / p.chunk : 1;
-  const int64_t base = ((int64_t)b * p.H + h) * p.n_chunks;
+  __syncthreads();
+  auto pair = [&](int k) { return staged ? s_ml[k] : p.ws_ml[base + k]; };
   float M = neg_inf();
-  for (int k = 0; k < ns; ++k) M = fmaxf(M, p.ws_ml[base + k].x);
+  for (int k = 0; k < ns; ++k) M = fmaxf(M, pair(k).x);
   float L = 0.f, A = 0.f;
-  for (int k = 0; k < ns; ++k) {
-    const float2 ml = p.ws_ml[base + k];
-    const float w = (ml.x > neg_inf()) ? fast_exp2(ml.x - M) : 0.f;
-    L = fmaf(ml.y, w, L);
-    A = fmaf(p.ws_acc[(base + k) * D + d], w, A);
+#pragma unroll
+  for (int k = 0; k < kMergeAhead; ++k) {
+    if (k < ns) {
+      const float2 ml = pair(k);
+      const float w = (ml.x > neg_inf()) ? fast_exp2(ml.x - M) : 0.f;
+      L = fmaf(ml.y, w, L);
+      A = fmaf(ahead[k], w, A);
+    }
+  }
+  for (int k0 = kMergeAhead; k0 < ns; k0 += kMergeAhead) {   // long requests: eight rows per trip
+    float rows[kMergeAhead];
+#pragma unroll
+    for (int j = 0; j < kMergeAhead; ++j) rows[j] = k0 + j < ns ? p.ws_acc[(base + k0 + j) * D + d] : 0.f;
+#pragma unroll
+    for (int j = 0; j < kMergeAhead; ++j) {
+      if (k0 + j < ns) {
+        const float2 ml = pair(k0 + j);
+        const float w = (ml.x > neg_inf()) ? fast_exp2(ml.x - M) : 0.f;
+        L = fmaf(ml.y, w, L);
+        A = fmaf(rows[j], w, A);
+      }
+    }
   }
   store_out<T>(p, b, h, d, L > 0.f ? A / L : 0.f);
   if (d == 0 && p.lse) p.lse[(int64_t)b * p.H + h] = L > 0.f ? (M + log2f(L)) * kLn2 : neg_inf();
@@ -485,14 +517,14 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   int chunk = 256;
   if (max_selected <= kMaxChunk && (units >= sms || max_selected <= 256)) chunk = kMaxChunk;
   else while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
-  if (shares_rows(d) && max_selected > kMaxChunk) {
+  if (shares_rows(d)) {
     // The row-sharing kernel leaves G triples per chunk, its blocks stream (a ring of tiles per warp) and two of
     // them fit an SM: about one block per resident slot, i.e. as few chunks as keep the SMs busy (measured,
     // B*H_kv = 64..256, context 8192: within 3 % of the best split for groups of 4, 8 and 16 heads).
     const long long target = sms * 2;
     long long n = target / units;                              // rounded down: never one block over a full wave
     n = std::max<long long>(1, std::min<long long>(n, (max_selected + 255) / 256));
-    chunk = std::max(chunk, (int)(((max_selected + n - 1) / n + 63) / 64 * 64));
+    chunk = (int)(((max_selected + n - 1) / n + 63) / 64 * 64);
   }
   int n_chunks = (max_selected + chunk - 1) / chunk;
   if (n_chunks == 1) chunk = (max_selected + 31) / 32 * 32;

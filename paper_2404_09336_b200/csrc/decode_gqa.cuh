@@ -82,7 +82,8 @@ constexpr int kStagedSmemBytes = kWarps * kStagedWarpBytes;   // 96 KB: two bloc
 // system rewards (full context at 32 query heads over 8 / 4 / 2 K/V heads: 6.9 / 6.3 / 5.4 TB/s with windows
 // of 256 rows, 6.7 / 6.2 / 5.4 with 512, 6.5 / 6.0 / 5.4 with 1024, 6.3 / 5.8 / 5.2 without windows), but each
 // meeting lets the ring run empty once (windows of 64 rows: 5.7 / 5.2 / 4.6 TB/s).
-constexpr int kStagedWindow = 512;                       // list entries staged at a time
+constexpr int kStagedWindow = 512;                       // list entries staged at a time ...
+constexpr int kStagedShortList = 1024;                   // ... unless the whole chunk fits this many: then one window
 constexpr int kStagedDenseWindow = 256;                  // full context: rows between two meetings of the warps
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -124,7 +125,7 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   static_assert(kWarps * kLiveHeads * (D + kGqaPad) * 4 <= kStagedSmemBytes, "the combine reuses the ring");
 
   extern __shared__ __align__(128) unsigned char s_ring[];
-  __shared__ int32_t s_idx[kSparse ? kStagedWindow : 1];
+  __shared__ int32_t s_idx[kSparse ? kStagedShortList : 1];
   __shared__ __align__(128) unsigned char s_qtile[kGqaHeads * 256];   // Q of the group, swizzled like a row tile
   __shared__ float s_m[kWarps][kLiveHeads], s_l[kWarps][kLiveHeads];
   __shared__ typename std::conditional<kMode == kSpans, SpanRuns, int>::type s_runs;
@@ -138,6 +139,28 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   grid_dependency_wait();
   if (p.early_release) grid_launch_dependents();
 
+  // One round trip for everything that does not depend on the list length: the first kStagedShortList list
+  // entries of the chunk (within the host's bound, so inside the caller's row) and the group's query rows.
+  constexpr int kAhead = kStagedShortList / kThreads;
+  int32_t ahead[kAhead];
+  const bool listed = kMode == kIndex && p.index != nullptr;
+  if (listed) {
+    const int32_t* row = p.index + (int64_t)b * p.index_stride + start;
+#pragma unroll
+    for (int jj = 0; jj < kAhead; ++jj) {
+      const int i = tid + jj * kThreads;
+      ahead[jj] = (i < p.chunk && start + i < p.max_selected) ? __ldg(row + i) : -1;
+    }
+  }
+  uint4 q_lo = make_uint4(0u, 0u, 0u, 0u), q_hi = make_uint4(0u, 0u, 0u, 0u);
+  {
+    const int row = tid >> 3, c0 = (tid & 7) * 2;
+    if (row < G) {
+      const T* src = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)(kvh * G + row) * p.q_sh + 8 * c0;
+      q_lo = ld_stream_16B(src);
+      q_hi = ld_stream_16B(src + 8);
+    }
+  }
   uint32_t flags = 0;
   int n, c;
   request_sizes(p, b, n, c, flags);
@@ -166,31 +189,40 @@ decode_partial_gqa_kernel(const DecodeParams p) {
       }
       return;
     }
-    const int32_t* row = p.index ? p.index + (int64_t)b * p.index_stride + start + w0 : nullptr;
-    for (int i = tid; i < wn; i += kThreads) {
-      int v = row ? __ldg(row + i) : start + w0 + i;
+    // position -> what the tile loop uses: -1 for an entry outside the context, the pool row for a paged cache
+    auto checked = [&](int v) {
       if (v < 0 || v >= n) {
-        v = -1; flags |= SSA_DEV_BAD_INDEX;
-      } else if (p.page_table) {
-        const int page = __ldg(p.page_table + (int64_t)b * p.page_table_stride + (v >> p.page_shift));
-        if ((unsigned)page < (unsigned)p.n_pages) v = (page << p.page_shift) | (v & p.page_mask);
-        else { v = -1; flags |= SSA_DEV_BAD_INDEX; }
+        flags |= SSA_DEV_BAD_INDEX;
+        return -1;
       }
-      s_idx[i] = v;
+      if (p.page_table) {
+        const int page = __ldg(p.page_table + (int64_t)b * p.page_table_stride + (v >> p.page_shift));
+        if ((unsigned)page < (unsigned)p.n_pages) return (page << p.page_shift) | (v & p.page_mask);
+        flags |= SSA_DEV_BAD_INDEX;
+        return -1;
+      }
+      return v;
+    };
+    if (listed && w0 == 0) {                             // the entries requested ahead cover any first window
+#pragma unroll
+      for (int jj = 0; jj < kAhead; ++jj) {
+        const int i = tid + jj * kThreads;
+        if (i < wn) s_idx[i] = checked(ahead[jj]);
+      }
+      return;
     }
+    const int32_t* row = listed ? p.index + (int64_t)b * p.index_stride + start + w0 : nullptr;
+    for (int i = tid; i < wn; i += kThreads)             // no list: the position itself (a paged full context)
+      s_idx[i] = checked(row ? __ldg(row + i) : start + w0 + i);
   };
-  if (kSparse) stage_window(0, min(cnt, kStagedWindow));
+  // a list chunk of up to kStagedShortList entries is one window (no meeting in mid-chunk); longer ones go by 512
+  const int window = kSparse ? (cnt <= kStagedShortList ? kStagedShortList : kStagedWindow) : kStagedDenseWindow;
+  if (kSparse) stage_window(0, min(cnt, window));
   // the group's query rows -> shared memory (rows of heads that do not exist are zero)
   {
     const int row = tid >> 3, c0 = (tid & 7) * 2;
-    uint4 a = make_uint4(0u, 0u, 0u, 0u), c2 = make_uint4(0u, 0u, 0u, 0u);
-    if (row < G) {
-      const T* src = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)(kvh * G + row) * p.q_sh + 8 * c0;
-      a = ld_stream_16B(src);
-      c2 = ld_stream_16B(src + 8);
-    }
-    *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0)) = a;
-    *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0 + 1)) = c2;
+    *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0)) = q_lo;
+    *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0 + 1)) = q_hi;
   }
   __syncthreads();
   // A fragments of Q for the eight k-steps: registers for the whole block's life
@@ -216,9 +248,8 @@ decode_partial_gqa_kernel(const DecodeParams p) {
 #pragma unroll
   for (int u = 0; u < 16; ++u) { o[u][0] = 0.f; o[u][1] = 0.f; o[u][2] = 0.f; o[u][3] = 0.f; }
 
-  constexpr int kWindow = kSparse ? kStagedWindow : kStagedDenseWindow;
-  for (int w0 = 0; w0 < cnt; w0 += kWindow) {
-    const int wn = min(kWindow, cnt - w0);
+  for (int w0 = 0; w0 < cnt; w0 += window) {
+    const int wn = min(window, cnt - w0);
     if (kSparse && w0 > 0) {
       __syncthreads();                                 // every warp is done with the previous window
       stage_window(w0, wn);

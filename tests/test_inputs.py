@@ -111,3 +111,15 @@ def test_shard_partitions_the_batch():
     assert np.array_equal(p.spans_of(0), wl.spans_of(g))
     assert np.array_equal(p.kv_bits_seq(0)[0], wl.kv_bits_seq(g)[0])
     assert np.array_equal(p.q_bits()[0], wl.q_bits()[g])
+
+
+def test_mixed_workload_replaces_every_kth_list_by_the_full_context():
+    base = inputs.make_config(2, B=9, H=2)
+    mixed = inputs.make_mixed(4, B=9, H=2)
+    assert np.array_equal(mixed.ctx_lens, base.ctx_lens) and mixed.seed == base.seed
+    for b in range(9):
+        if b % 4 == 0:
+            assert mixed.spans_of(b).tolist() == [[0, int(base.ctx_lens[b])]]
+        else:
+            assert mixed.spans_of(b).tolist() == base.spans_of(b).tolist()
+    assert mixed.selected_upper_bound() == int(base.ctx_lens[[0, 4, 8]].max())
