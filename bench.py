@@ -53,9 +53,10 @@ WORKLOAD_TEXT = {
     5: "cfg5 density sweep: B=32 H=32 D=128 ctx=8192 bf16",
 }
 
-# DRAM traffic of one launch of the dominant kernel at cfg 2 (dram__bytes_read.sum + dram__bytes_write.sum of
-# one ncu capture), valid only for the kernel source it was captured from.
-NCU_TRAFFIC = {"source_sha256_16": "3847ce96bbc6587b", "cfg": 2, "bytes_per_launch": 152399104}
+# DRAM traffic of one launch of the dominant kernel at cfg 2, the index-list kernel of the two-kernel step
+# (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture: 148 971 008 + 4 232 448), valid only for the
+# kernel sources it was captured from and for that form of the step.
+NCU_TRAFFIC = {"source_sha256_16": "6eb4a6ec37d5df8e", "cfg": 2, "bytes_per_launch": 153203456}
 
 
 def log(*a):
@@ -760,8 +761,8 @@ def run_ours(args):
         return
 
     kernel_us = main["kernel_us"]
-    traffic = NCU_TRAFFIC["bytes_per_launch"] if (args.cfg == NCU_TRAFFIC["cfg"] and
-                                                  kernel_source_hash() == NCU_TRAFFIC["source_sha256_16"]) else None
+    traffic = NCU_TRAFFIC["bytes_per_launch"] if (args.cfg == NCU_TRAFFIC["cfg"] and main["path"] == "index + attention"
+                                                  and kernel_source_hash() == NCU_TRAFFIC["source_sha256_16"]) else None
     kernel_name = ("decode_partial_kernel<spans> (ssa_decode_attn_spans)" if main["path"] == "one kernel"
                    else "decode_partial_kernel<index> (ssa_decode_attn_sparse)")
     roofline = {"bound": "hbm", "kernel": kernel_name,
