@@ -444,7 +444,11 @@ int32_t ssa_decode_attn_blockmask(const ssa_attn_desc* desc, const void* q, cons
  * library that read / write the host arena across the bus (when span_offsets,
  * spans and ctx_lens lie inside the input arena, the copy in is done by extra
  * blocks of the index kernel, whose other blocks read the span lists from the
- * host arena meanwhile).  For the few
+ * host arena meanwhile; where, besides, the query rows are the head or the
+ * tail of the input arena and every request is served by one thread block per
+ * head, each attention block fetches its own query row across the bus while it
+ * starts up and writes the device copy itself, so that most of the input
+ * bytes travel during the attention kernel instead of in front of it).  For the few
  * hundred KB that change per decode step this is faster than a copy-engine
  * transfer, whose set-up time dominates at that size.  The host arenas must
  * then be page-locked memory that the device addresses under the same pointer

@@ -52,6 +52,8 @@ constexpr int kMaskChunk = 512;        // positions a block expands from bitmask
 enum { kDense = 0, kIndex = 1, kBlockMask = 2, kSpans = 3 };
 
 struct DecodeParams {
+  const void* q_host;       // kHostQ only: the query rows in page-locked host memory the device addresses; every
+                            // block fetches its own row across the bus and leaves a copy at q
   const void* q;
   const void* k;
   const void* v;
@@ -146,10 +148,14 @@ __device__ __forceinline__ void zero_piece(Piece& r) {
 
 // kPaged (index lists only): positions are translated through the page table while they are staged, and a
 // missing list stands for 0, 1, 2, ...; kept out of the unpaged instantiations so that they stay as they are.
-template <typename T, int D, int kMode, bool kAligned32, bool kPaged = false>
+// kHostQ (index lists, one chunk per request): the query rows are still in page-locked host memory.  Each block
+// asks for its row (D/8 threads, 16 bytes each) before anything else, so that the trip across the bus overlaps
+// the block's start-up, shares it through shared memory and writes the device copy the caller expects at q.
+template <typename T, int D, int kMode, bool kAligned32, bool kPaged = false, bool kHostQ = false>
 __global__ void __launch_bounds__(kThreads, SSA_MIN_BLOCKS)
 decode_partial_kernel(const DecodeParams p) {
   static_assert(!kPaged || kMode == kIndex, "a paged cache is read through staged positions");
+  static_assert(!kHostQ || (kMode == kIndex && !kPaged), "host-resident queries: plain index lists only");
   using TQ = typename Storage<T>::Query;              // type of the query rows and of a stored output
   constexpr bool kFp8 = kIsFp8<T>;
   constexpr int kU = kFp8 ? 2 * SSA_U : SSA_U;        // 8-bit pieces are half as large: twice as many in flight
@@ -168,6 +174,7 @@ decode_partial_kernel(const DecodeParams p) {
   __shared__ int s_wcount[kWarps];
   __shared__ typename std::conditional<kMode == kSpans, SpanRuns, int>::type s_runs;
   __shared__ typename std::conditional<kMode == kSpans, WarpRuns, int>::type s_wruns[kMode == kSpans ? kWarps : 1];
+  __shared__ uint4 s_qrow[kHostQ ? D / 8 : 1];
 
   const int chunk_id = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -176,6 +183,13 @@ decode_partial_kernel(const DecodeParams p) {
 
   grid_dependency_wait();
   if (p.early_release) grid_launch_dependents();      // small grid: let the next kernel's blocks move in now
+
+  uint4 q_word = make_uint4(0u, 0u, 0u, 0u);          // kHostQ: this thread's 16 bytes of the query row
+  if constexpr (kHostQ) {
+    if (tid < D / 8)
+      q_word = *(reinterpret_cast<const uint4*>(reinterpret_cast<const TQ*>(p.q_host) + (int64_t)b * p.q_sb +
+                                                (int64_t)h * p.q_sh) + tid);
+  }
 
   // Everything the block needs before it can request cache rows is loaded
   // here in one go: sizes, its slice of the index list, the query row.
@@ -196,7 +210,7 @@ decode_partial_kernel(const DecodeParams p) {
     }
   }
   Piece qraw;                                         // re-read by every warp and chunk of the head: plain L2 policy
-  {
+  if constexpr (!kHostQ) {
     const char* qp = reinterpret_cast<const char*>(
         reinterpret_cast<const TQ*>(p.q) + (int64_t)b * p.q_sb + (int64_t)h * p.q_sh + col * 16);
     const uint4 a = ld_stream_16B(qp), c4 = ld_stream_16B(qp + 16);
@@ -322,6 +336,18 @@ decode_partial_kernel(const DecodeParams p) {
   const char* vbase = reinterpret_cast<const char*>(
       reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)(h / p.kv_group) * p.v_sh + col * 16);
 
+  if constexpr (kHostQ) {
+    // the row has crossed the bus by now (or is about to): share it, and leave the device copy
+    if (tid < D / 8) {
+      s_qrow[tid] = q_word;
+      *(reinterpret_cast<uint4*>(const_cast<TQ*>(reinterpret_cast<const TQ*>(p.q)) + (int64_t)b * p.q_sb +
+                                 (int64_t)h * p.q_sh) + tid) = q_word;
+    }
+    __syncthreads();                                  // one chunk per request: every block gets here
+    const uint4 a = s_qrow[2 * col], c4 = s_qrow[2 * col + 1];
+    qraw.w[0] = a.x; qraw.w[1] = a.y; qraw.w[2] = a.z; qraw.w[3] = a.w;
+    qraw.w[4] = c4.x; qraw.w[5] = c4.y; qraw.w[6] = c4.z; qraw.w[7] = c4.w;
+  }
   float2 q2[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -601,7 +627,13 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   if (!share) {
     constexpr bool kWide = !kFp8;                       // 8-bit rows are read in 16-byte pieces: one instantiation
     const bool a32 = kWide && aligned32;
-    if (mode == kIndex && p.page_table)
+    if constexpr (!kFp8) {
+      if (p.q_host)                                     // run() has checked: index lists, one chunk, no paging
+        kernel = a32 ? decode_partial_kernel<T, D, kIndex, true, false, true>
+                     : decode_partial_kernel<T, D, kIndex, false, false, true>;
+    }
+    if (p.q_host) {
+    } else if (mode == kIndex && p.page_table)
       kernel = a32 ? decode_partial_kernel<T, D, kIndex, kWide, true> : decode_partial_kernel<T, D, kIndex, false, true>;
     else if (mode == kIndex)
       kernel = a32 ? decode_partial_kernel<T, D, kIndex, kWide> : decode_partial_kernel<T, D, kIndex, false>;
@@ -647,7 +679,7 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
                    const int32_t* counts, int32_t max_selected, void* out, float* lse,
                    void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream, int mode,
                    const BlockList* bl = nullptr, const ssa_paging* pg = nullptr,
-                   const SpanLists* sl = nullptr) {
+                   const SpanLists* sl = nullptr, const void* q_host = nullptr) {
   // a paged cache is read through the staged-positions path; without a list the positions are 0 .. ctx_len-1
   const bool dense_paged = pg && mode == kDense;
   if (dense_paged) mode = kIndex;
@@ -692,7 +724,11 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   }
   if (!ws || ws_bytes < pl.total_bytes + (mode == kSpans ? counts_bytes(d) : 0)) return SSA_ERR_WORKSPACE;
 
+  if (q_host && !(mode == kIndex && !pg && !dense_paged && pl.n_chunks == 1 && !shares_rows(d) &&
+                  d->kv_dtype != SSA_FP8_E4M3 && aligned16(q_host)))
+    return SSA_ERR_UNSUPPORTED;
   DecodeParams p;
+  p.q_host = q_host;
   p.span_offsets = mode == kSpans ? sl->span_offsets : nullptr;
   p.spans = mode == kSpans ? reinterpret_cast<const int2*>(sl->spans) : nullptr;
   p.span_cap = mode == kSpans ? sl->span_cap : 0;
@@ -750,6 +786,26 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
 }
 
 int32_t one_kernel_span_limit() { return kDirectSpans; }
+
+// ssa_decode_attn_sparse with the query rows still in page-locked host memory that the device addresses (q_host,
+// laid out like q): every block fetches its own row across the bus and writes the device copy at q.  Offered
+// where host_queries_pay() says so.
+int32_t decode_attn_sparse_host_queries(const ssa_attn_desc* desc, void* q, const void* q_host, const void* k_cache,
+                                        const void* v_cache, const int32_t* ctx_lens, const int32_t* index,
+                                        int32_t index_stride, const int32_t* counts, int32_t max_selected, void* out,
+                                        float* lse, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                        void* stream) {
+  if (!q_host) return SSA_ERR_NULL;
+  return run(desc, q, k_cache, v_cache, ctx_lens, index, index_stride, counts, max_selected, out, lse, workspace,
+             workspace_bytes, dev_status, stream, kIndex, nullptr, nullptr, nullptr, q_host);
+}
+
+// One chunk per request (every row then crosses the bus once), multi-head 16-bit cache.
+bool host_queries_pay(const ssa_attn_desc* d, int32_t max_selected) {
+  Plan pl;
+  if (!d || check_desc(d) != SSA_OK || !make_plan(d, max_selected, &pl)) return false;
+  return pl.n_chunks == 1 && !shares_rows(d) && d->kv_dtype != SSA_FP8_E4M3;
+}
 
 // Every block of the span-list kernel repeats the merge of its request's spans (about a microsecond per wave
 // of blocks when a warp can do it alone), the index kernel does it once per request but costs a launch of its

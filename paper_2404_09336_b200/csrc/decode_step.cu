@@ -90,11 +90,30 @@ extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s,
                                s->workspace, s->workspace_bytes, s->dev_status, stream);
     if (rc != SSA_OK) return rc;
   } else {
+  const void* q_host = nullptr;                // set: the attention kernel fetches the query rows itself
   if (fused_fetch) {
-    // the span lists are part of what is fetched: expand them straight from the host arena while the same
-    // launch copies the arena in
+    // The span lists are part of what is fetched: expand them straight from the host arena while the same
+    // launch copies the arena in.  Where the query rows are the head or the tail of the arena and every request
+    // is served by one thread block per head, that copy leaves them out: each attention block then fetches its
+    // own row across the bus while it starts up (and writes the device copy), so the bulk of the input bytes
+    // travels during the attention kernel instead of in front of it.
+    const char* arena = static_cast<const char*>(s->dev_in);
+    const char* q_dev = static_cast<const char*>(s->q);
+    const size_t q_bytes = ((size_t)(desc->B - 1) * desc->q_stride_b + (size_t)(desc->H - 1) * desc->q_stride_h +
+                            desc->D) * 2;
+    size_t skip_head = 0, skip_tail = 0;
+    if (host_twin(s->q) && q_bytes % 16 == 0 && q_bytes <= s->in_bytes && ssa::host_queries_pay(desc, s->max_selected)) {
+      if (q_dev == arena) skip_head = q_bytes;
+      else if (q_dev + q_bytes == arena + s->in_bytes) skip_tail = q_bytes;
+    }
+    if (skip_head + skip_tail > 0 && skip_head + skip_tail < s->in_bytes)
+      q_host = static_cast<const char*>(s->host_in) + (q_dev - arena);
+    else
+      skip_head = skip_tail = 0;
     rc = ssa::fetch_and_index(h_off, h_spans, h_ctx, desc->B, s->index, s->index_stride, s->counts, s->dev_status,
-                              s->dev_in, s->host_in, s->in_bytes, st);
+                              static_cast<char*>(s->dev_in) + skip_head,
+                              static_cast<const char*>(s->host_in) + skip_head,
+                              s->in_bytes - skip_head - skip_tail, st);
     if (rc != SSA_OK) return rc;
   } else {
     if (s->host_in) {
@@ -109,9 +128,14 @@ extern "C" int32_t ssa_decode_step(const ssa_attn_desc* desc, const ssa_step* s,
                             s->counts, s->dev_status, stream);
     if (rc != SSA_OK) return rc;
   }
-  rc = ssa_decode_attn_sparse(desc, s->q, s->k_cache, s->v_cache, s->ctx_lens, s->index, s->index_stride,
-                              s->counts, s->max_selected, s->out, s->lse, s->workspace, s->workspace_bytes,
-                              s->dev_status, stream);
+  if (q_host)
+    rc = ssa::decode_attn_sparse_host_queries(desc, const_cast<void*>(s->q), q_host, s->k_cache, s->v_cache,
+                                              s->ctx_lens, s->index, s->index_stride, s->counts, s->max_selected,
+                                              s->out, s->lse, s->workspace, s->workspace_bytes, s->dev_status, stream);
+  else
+    rc = ssa_decode_attn_sparse(desc, s->q, s->k_cache, s->v_cache, s->ctx_lens, s->index, s->index_stride,
+                                s->counts, s->max_selected, s->out, s->lse, s->workspace, s->workspace_bytes,
+                                s->dev_status, stream);
   if (rc != SSA_OK) return rc;
   }
   if (s->host_out) {

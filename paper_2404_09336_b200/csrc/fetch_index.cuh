@@ -21,4 +21,13 @@ int32_t spans_to_index_capped(const int32_t* span_offsets, const int32_t* spans,
 int32_t one_kernel_span_limit();
 bool one_kernel_step_pays(const ssa_attn_desc* desc, int32_t max_selected, int32_t max_spans, size_t workspace_bytes);
 
+// Defined in decode_attn.cu, for ssa_decode_step with copies done by kernels: the attention call that fetches the
+// query rows itself (see there), and whether a step qualifies.
+int32_t decode_attn_sparse_host_queries(const ssa_attn_desc* desc, void* q, const void* q_host, const void* k_cache,
+                                        const void* v_cache, const int32_t* ctx_lens, const int32_t* index,
+                                        int32_t index_stride, const int32_t* counts, int32_t max_selected, void* out,
+                                        float* lse, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                        void* stream);
+bool host_queries_pay(const ssa_attn_desc* desc, int32_t max_selected);
+
 }  // namespace ssa
