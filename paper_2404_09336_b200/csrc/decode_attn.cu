@@ -336,33 +336,11 @@ decode_partial_kernel(const DecodeParams p) {
   const char* vbase = reinterpret_cast<const char*>(
       reinterpret_cast<const T*>(p.v) + (int64_t)b * p.v_sb + (int64_t)(h / p.kv_group) * p.v_sh + col * 16);
 
-  if constexpr (kHostQ) {
-    // the row has crossed the bus by now (or is about to): share it, and leave the device copy
-    if (tid < D / 8) {
-      s_qrow[tid] = q_word;
-      *(reinterpret_cast<uint4*>(const_cast<TQ*>(reinterpret_cast<const TQ*>(p.q)) + (int64_t)b * p.q_sb +
-                                 (int64_t)h * p.q_sh) + tid) = q_word;
-    }
-    __syncthreads();                                  // one chunk per request: every block gets here
-    const uint4 a = s_qrow[2 * col], c4 = s_qrow[2 * col + 1];
-    qraw.w[0] = a.x; qraw.w[1] = a.y; qraw.w[2] = a.z; qraw.w[3] = a.w;
-    qraw.w[4] = c4.x; qraw.w[5] = c4.y; qraw.w[6] = c4.z; qraw.w[7] = c4.w;
-  }
-  float2 q2[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    q2[i] = unpack2<TQ>(qraw.w[i]);
-    q2[i].x *= p.scale_log2;
-    q2[i].y *= p.scale_log2;
-  }
-  float m = neg_inf(), l = 0.f;
-  float2 acc[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) acc[i] = make_float2(0.f, 0.f);
-
-  for (int t = warp * kTileRows; t < cnt; t += kWarps * kTileRows) {
-    Piece kr[kU], vr[kU];
-    float s[kU];
+  // Requests the K and V rows of the warp's tile that starts at row t of the block; returns whether the tile needs
+  // the predicated path (a ragged tail or entries that were skipped).
+  Piece kr[kU], vr[kU];
+  float s[kU];
+  auto request_tile = [&](int t) -> bool {
     // full tiles without bad entries take the unpredicated path
     const bool checked = any_bad || (t + kTileRows > cnt);
     if (!checked) {
@@ -389,6 +367,46 @@ decode_partial_kernel(const DecodeParams p) {
           s[u] = neg_inf();                           // marks the row as masked
         }
       }
+    }
+    return checked;
+  };
+  bool pre_issued = false, pre_checked = false;
+  if constexpr (kHostQ) {
+    // the first tile's rows are requested before the block waits for its query row
+    if (warp * kTileRows < cnt) {
+      pre_checked = request_tile(warp * kTileRows);
+      pre_issued = true;
+    }
+    // the row has crossed the bus by now (or is about to): share it, and leave the device copy
+    if (tid < D / 8) {
+      s_qrow[tid] = q_word;
+      *(reinterpret_cast<uint4*>(const_cast<TQ*>(reinterpret_cast<const TQ*>(p.q)) + (int64_t)b * p.q_sb +
+                                 (int64_t)h * p.q_sh) + tid) = q_word;
+    }
+    __syncthreads();                                  // one chunk per request: every block gets here
+    const uint4 a = s_qrow[2 * col], c4 = s_qrow[2 * col + 1];
+    qraw.w[0] = a.x; qraw.w[1] = a.y; qraw.w[2] = a.z; qraw.w[3] = a.w;
+    qraw.w[4] = c4.x; qraw.w[5] = c4.y; qraw.w[6] = c4.z; qraw.w[7] = c4.w;
+  }
+  float2 q2[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    q2[i] = unpack2<TQ>(qraw.w[i]);
+    q2[i].x *= p.scale_log2;
+    q2[i].y *= p.scale_log2;
+  }
+  float m = neg_inf(), l = 0.f;
+  float2 acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = make_float2(0.f, 0.f);
+
+  for (int t = warp * kTileRows; t < cnt; t += kWarps * kTileRows) {
+    bool checked;
+    if (kHostQ && pre_issued) {                         // the warp's first tile is already on its way
+      checked = pre_checked;
+      pre_issued = false;
+    } else {
+      checked = request_tile(t);
     }
     float mt = neg_inf();
 #pragma unroll
