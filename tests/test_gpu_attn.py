@@ -7,7 +7,7 @@ from oracle import ssa_oracle as O
 from paper_2404_09336_b200 import inputs, ssa
 from paper_2404_09336_b200.runner import DecodeStep
 
-from gpu_util import Problem, random_bits, run_index
+from gpu_util import DEV, Problem, random_bits, run_index
 from parity import assert_parity
 
 pytestmark = pytest.mark.gpu
@@ -754,3 +754,50 @@ def test_one_long_context_with_hundreds_of_spans():
     ref_d, ref_lse_d = O.decode_attn_dense(p.q_bits, p.k_bits, p.v_bits, [T], scale_of(D), "f16")
     assert_parity(out_d, ref_d, False, "long context, dense")
     np.testing.assert_allclose(lse_d, ref_lse_d, rtol=1e-5, atol=1e-5)
+
+
+@pytest.mark.parametrize("order", ["q first", "q last", "q in the middle"])
+def test_host_driven_step_wherever_the_query_rows_sit_in_the_input_arena(order):
+    """SSA_STEP_COPY_BY_KERNEL with hand-laid arenas: with the query rows at the head or the tail of the arena the
+    attention blocks fetch them from the pinned copy themselves (one chunk per request here); in the middle the
+    whole arena is fetched in front of the kernels.  Either way: the oracle's output, and the device arena ends up
+    a copy of the host arena."""
+    wl = inputs.make_config(2, B=5, H=4)
+    B, H, D = wl.B, wl.H, wl.D
+    n_spans = len(wl.spans)
+    sizes = {"q": B * H * D * 2, "ctx": B * 4, "offs": (B + 1) * 4, "spans": n_spans * 8}
+    pad = lambda n: (n + 255) // 256 * 256
+    names = {"q first": ["q", "ctx", "offs", "spans"], "q last": ["ctx", "offs", "spans", "q"],
+             "q in the middle": ["ctx", "q", "offs", "spans"]}[order]
+    at, total = {}, 0
+    for i, name in enumerate(names):
+        at[name] = total
+        total += sizes[name] if i == len(names) - 1 else pad(sizes[name])   # nothing behind the last tensor
+    total = (total + 15) // 16 * 16
+    h_in = torch.zeros(total, dtype=torch.uint8).pin_memory()
+    view = lambda buf, name, dt, shape: buf[at[name]:at[name] + sizes[name]].view(dt).view(shape)
+    view(h_in, "q", torch.bfloat16, (B, H, D)).copy_(torch.from_numpy(wl.q_bits().view(np.int16)).view(torch.bfloat16))
+    view(h_in, "ctx", torch.int32, (B,)).copy_(torch.from_numpy(wl.ctx_lens.copy()))
+    view(h_in, "offs", torch.int32, (B + 1,)).copy_(torch.from_numpy(wl.span_offsets.copy()))
+    view(h_in, "spans", torch.int32, (n_spans, 2)).copy_(torch.from_numpy(np.ascontiguousarray(wl.spans)))
+    d_in = torch.full((total,), 0xAB, dtype=torch.uint8, device=DEV)
+    q = view(d_in, "q", torch.bfloat16, (B, H, D))
+    ctx, offs = view(d_in, "ctx", torch.int32, (B,)), view(d_in, "offs", torch.int32, (B + 1,))
+    spans = view(d_in, "spans", torch.int32, (n_spans, 2))
+    ds = DecodeStep(wl, out_dtype=torch.float32)              # the cache, and buffers to borrow
+    h_out = torch.zeros(ds.counts.numel() * 4 + 256, dtype=torch.uint8).pin_memory()
+    ds.index.fill_(-7)
+    ds.status.zero_()
+    desc = ssa.make_desc(q, ds.k, ds.v, ds.out)
+    st = ssa.make_step(offs, spans, ctx, ds.index, ds.counts, q, ds.k, ds.v, ds.max_selected, ds.out, ds.lse,
+                       ds.workspace, ds.status, host_in=h_in, dev_in=d_in, copy_by_kernel=True, max_spans=ds.max_spans)
+    for _ in range(2):
+        ds.out.fill_(3.0)
+        ssa.decode_step(desc, st)
+        torch.cuda.synchronize()
+        assert torch.equal(d_in.cpu(), h_in)                  # every input byte arrived on the device
+        assert int(ds.status.item()) == 0
+    index, counts, _ = O.spans_to_index_batch(wl.span_offsets, wl.spans, wl.ctx_lens, ds.index_stride)
+    assert ds.counts.cpu().numpy().tolist() == counts.tolist()
+    ref, _ = O.decode_attn_sparse(wl.q_bits(), *wl.kv_bits(), wl.ctx_lens, index, counts, scale_of(D), wl.dtype)
+    assert_parity(ds.out_f64(), ref, False, order)
