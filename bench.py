@@ -812,7 +812,7 @@ def run_ours(args):
 
     if world == 1:
         sweep = []
-        want = {"auto": [3, 4, 5], "all": [1, 3, 4, 5], "none": []}[args.sweep]
+        want = {"auto": [1, 3, 4, 5], "all": [1, 3, 4, 5], "none": []}[args.sweep]
         sweep_steps, sweep_regions = max(20, min(steps, 100)), max(3, min(regions, 9))
         del ds
         torch.cuda.empty_cache()
