@@ -426,7 +426,7 @@ def measure(torch, ssa, timer, ds, steps, warmup, regions, pieces=True):
     # to back (CUDA events around the region on the launching stream; region / launches).  Where the lists span
     # several chunks the call's small second pass rides along, so the figure errs on the long side.
     ds.build_index()
-    attend = ds.attend_spans if one_kernel else ds.attend_sparse
+    attend = (lambda: ds.step(kernels="one")) if one_kernel else ds.attend_sparse   # one kernel: the step is the call
     for i in range(3):
         attend()
     res["kernel_us"] = timer.median_us(rotating(attend), steps, regions)
