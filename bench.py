@@ -849,6 +849,8 @@ def run_ours(args):
             roofline["read_stream_how"] = ("best rate of this library's full-context kernel in this run (a read-only "
                                            "stream; the measured peak above is a copy, which a read-only stream exceeds)")
             roofline["frac_of_read_stream"] = round(roofline["achieved"] / read_peak, 4)
+            for e in roofline["by_config"]:            # no workload exceeds this denominator
+                e["frac_of_read_stream"] = round(e["bytes"] / e["kernel_us"] / 1e3 / read_peak, 4)
         five = [r for r in sweep if r["workload"].startswith("cfg5")]
         line["crossover_density"] = next((r["density"] for r in five if r["speedup_vs_dense"] < 1.0), None)
         if args.sweep != "none":
