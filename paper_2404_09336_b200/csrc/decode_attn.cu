@@ -78,6 +78,7 @@ struct DecodeParams {
   uint32_t k_row_bytes, v_row_bytes;   // token stride of the cache in bytes
   int32_t H, max_ctx, index_stride, max_selected, chunk, n_chunks, out_f32, early_release;
   int32_t kv_group;         // query heads per K/V head (1: multi-head attention)
+  int32_t gqa_wide;         // row-sharing kernel with eight warps per block
   // paged cache (page_table != nullptr): logical position t of request b is row
   // page_table[b * page_table_stride + (t >> page_shift)] << page_shift | (t & page_mask) of the pool
   const int32_t* page_table;
@@ -539,7 +540,7 @@ namespace ssa {
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
-struct Plan { int chunk, n_chunks; size_t acc_bytes, total_bytes; };
+struct Plan { int chunk, n_chunks; size_t acc_bytes, total_bytes; bool wide; };   // wide: eight-warp row-sharing blocks
 
 // Grouped query heads go to the kernel that reads a K/V row once for the whole group.
 static bool shares_rows(const ssa_attn_desc* d) {
@@ -561,7 +562,14 @@ static bool make_plan(const ssa_attn_desc* d, int max_selected, Plan* pl) {
   int chunk = 256;
   if (max_selected <= kMaxChunk && (units >= sms || max_selected <= 256)) chunk = kMaxChunk;
   else while (chunk > 64 && units * ((max_selected + chunk - 1) / chunk) < want) chunk >>= 1;
-  if (shares_rows(d)) {
+  pl->wide = false;
+  if (shares_rows(d) && 2 * units > sms && units <= sms && max_selected <= 2048) {
+    // One unit for most SMs and a short list: the whole list is one eight-warp block's work, and the second pass
+    // (about 3 us in the stream) is not needed (32 query heads over 4 K/V heads, 32 requests, 819 rows: 15.2 vs
+    // 18.0 us).  With fewer units (2 K/V heads: 64) too many SMs would idle: 15.2 vs 14.4 us with four chunks.
+    pl->wide = true;
+    chunk = (max_selected + 63) / 64 * 64;
+  } else if (shares_rows(d)) {
     // The row-sharing kernel leaves G triples per chunk, its blocks stream (a ring of tiles per warp) and two of
     // them fit an SM: about one block per resident slot, i.e. as few chunks as keep the SMs busy (measured,
     // B*H_kv = 64..256, context 8192: within 3 % of the best split for groups of 4, 8 and 16 heads).
@@ -585,6 +593,7 @@ static bool make_plan_blockmask(const ssa_attn_desc* d, int block_size, int max_
   if (d->D != 64 && d->D != 128) return false;
   if (block_size != 32 && block_size != 64 && block_size != 128 && block_size != 256) return false;
   const long long units = (long long)d->B * d->H;
+  pl->wide = false;
   pl->chunk = kMaskChunk / block_size;
   pl->n_chunks = (max_blocks + pl->chunk - 1) / pl->chunk;
   pl->acc_bytes = ((size_t)units * pl->n_chunks * d->D * sizeof(float) + 255) / 256 * 256;
@@ -625,20 +634,30 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
   using TQ = typename Storage<T>::Query;
   constexpr bool kFp8 = kIsFp8<T>;
   size_t dynamic_smem = 0;
+  unsigned block_threads = kThreads;
   bool share = false;
   if constexpr (!kFp8) {                                // the row-sharing kernel feeds 16-bit rows to the tensor cores
     share = D == 128 && p.kv_group >= 2 && p.kv_group <= kGqaHeads && mode != kBlockMask;
     if (share) {
       grid.y = (unsigned)(p.H / p.kv_group);            // one block per K/V head
       const bool hi = p.kv_group > 8;
-      if (mode == kIndex)
+      constexpr int kW8 = kGqaWideWarps;
+      if (p.gqa_wide) {
+        if (mode == kIndex)
+          kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true, kW8> : decode_partial_gqa_kernel<T, kIndex, false, kW8>;
+        else if (mode == kSpans)
+          kernel = hi ? decode_partial_gqa_kernel<T, kSpans, true, kW8> : decode_partial_gqa_kernel<T, kSpans, false, kW8>;
+        else
+          kernel = hi ? decode_partial_gqa_kernel<T, kDense, true, kW8> : decode_partial_gqa_kernel<T, kDense, false, kW8>;
+        block_threads = kW8 * 32;
+      } else if (mode == kIndex)
         kernel = hi ? decode_partial_gqa_kernel<T, kIndex, true> : decode_partial_gqa_kernel<T, kIndex, false>;
       else if (mode == kSpans)
         kernel = hi ? decode_partial_gqa_kernel<T, kSpans, true> : decode_partial_gqa_kernel<T, kSpans, false>;
       else
         kernel = hi ? decode_partial_gqa_kernel<T, kDense, true> : decode_partial_gqa_kernel<T, kDense, false>;
-      dynamic_smem = kStagedSmemBytes;
-      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStagedSmemBytes) != cudaSuccess)
+      dynamic_smem = (size_t)(block_threads / 32) * kStagedWarpBytes;
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynamic_smem) != cudaSuccess)
         return SSA_ERR_CUDA;
     }
   }
@@ -663,7 +682,7 @@ static int32_t launch(const DecodeParams& p, int B, int mode, bool aligned32, cu
       kernel = a32 ? decode_partial_kernel<T, D, kDense, kWide> : decode_partial_kernel<T, D, kDense, false>;
   }
   if (ev_b) cudaEventRecord(ev_b, st);
-  cudaError_t err = launch_pdl_smem(kernel, grid, dim3(kThreads), dynamic_smem, st, p);
+  cudaError_t err = launch_pdl_smem(kernel, grid, dim3(block_threads), dynamic_smem, st, p);
   if (ev_e) cudaEventRecord(ev_e, st);
   if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SSA_ERR_CUDA;
   int launches = 1;
@@ -782,6 +801,7 @@ static int32_t run(const ssa_attn_desc* d, const void* q, const void* k, const v
   p.H = d->H; p.max_ctx = d->max_ctx;
   p.index_stride = index_stride; p.max_selected = max_selected;
   p.chunk = pl.chunk; p.n_chunks = pl.n_chunks;
+  p.gqa_wide = pl.wide ? 1 : 0;
   p.out_f32 = d->out_dtype == SSA_F32;
   // A grid of a few waves releases the next kernel at once (its blocks wait on
   // chip instead of being launched after the drain); a long grid does so only

@@ -76,7 +76,8 @@ constexpr int kGqaPad = 4;              // floats of padding per head row of the
 constexpr int kStagedDepth = 3;                          // tiles per warp in the ring
 constexpr int kStagedTileBytes = kGqaRows * 256;         // one tensor's tile
 constexpr int kStagedWarpBytes = kStagedDepth * 2 * kStagedTileBytes;
-constexpr int kStagedSmemBytes = kWarps * kStagedWarpBytes;   // 96 KB: two blocks per SM
+constexpr int kStagedSmemBytes = kWarps * kStagedWarpBytes;   // four-warp blocks: 96 KB, two blocks per SM
+constexpr int kGqaWideWarps = 8;                         // eight-warp blocks (192 KB, one per SM) for short lists of few units
 // A chunk is worked through in windows: the block's warps meet at every window's end (and, for lists, stage
 // the next window's positions).  Meeting often keeps the four warps on neighbouring rows, which the memory
 // system rewards (full context at 32 query heads over 8 / 4 / 2 K/V heads: 6.9 / 6.3 / 5.4 TB/s with windows
@@ -114,15 +115,18 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int chunk) {
   return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4));
 }
 
-template <typename T, int kMode, bool kHi>
-__global__ void __launch_bounds__(kThreads, 2)
+// kW: warps per block.  Four is the rule (two blocks per SM).  Eight serve launches with at most one unit (request x
+// K/V head) per SM and short lists: a whole list is then one block's work - no second pass - and eight warps stream it.
+template <typename T, int kMode, bool kHi, int kW = kWarps>
+__global__ void __launch_bounds__(kW * 32, kW == kWarps ? 2 : 1)
 decode_partial_gqa_kernel(const DecodeParams p) {
+  constexpr int kWarps = kW, kThreads = kW * 32;      // hide the library-wide four-warp constants in here
   constexpr int D = 128;
   constexpr bool kSparse = kMode != kDense;
   constexpr int kLiveHeads = kHi ? 16 : 8;
   static_assert(kMode == kDense || kMode == kIndex || kMode == kSpans,
                 "blocked lists take the one-head-per-block kernel");
-  static_assert(kWarps * kLiveHeads * (D + kGqaPad) * 4 <= kStagedSmemBytes, "the combine reuses the ring");
+  static_assert(kLiveHeads * (D + kGqaPad) * 4 <= kStagedWarpBytes, "the combine reuses the ring");
 
   extern __shared__ __align__(128) unsigned char s_ring[];
   __shared__ int32_t s_idx[kSparse ? kStagedShortList : 1];
@@ -154,7 +158,7 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   }
   uint4 q_lo = make_uint4(0u, 0u, 0u, 0u), q_hi = make_uint4(0u, 0u, 0u, 0u);
   {
-    const int row = tid >> 3, c0 = (tid & 7) * 2;
+    const int row = tid >> 3, c0 = (tid & 7) * 2;     // 16 rows x 8 threads; further threads have no part
     if (row < G) {
       const T* src = reinterpret_cast<const T*>(p.q) + (int64_t)b * p.q_sb + (int64_t)(kvh * G + row) * p.q_sh + 8 * c0;
       q_lo = ld_stream_16B(src);
@@ -219,7 +223,7 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   const int window = kSparse ? (cnt <= kStagedShortList ? kStagedShortList : kStagedWindow) : kStagedDenseWindow;
   if (kSparse) stage_window(0, min(cnt, window));
   // the group's query rows -> shared memory (rows of heads that do not exist are zero)
-  {
+  if (tid < kGqaHeads * 8) {
     const int row = tid >> 3, c0 = (tid & 7) * 2;
     *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0)) = q_lo;
     *reinterpret_cast<uint4*>(s_qtile + tile_offset(row, c0 + 1)) = q_hi;
@@ -409,6 +413,7 @@ decode_partial_gqa_kernel(const DecodeParams p) {
   }
   __syncthreads();
   // thread d finishes dim d of every head
+  if (tid >= D) return;
   for (int i = 0; i < G; ++i) {
     const int h = kvh * G + i;
     float M = neg_inf();
